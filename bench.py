@@ -1,0 +1,414 @@
+#!/usr/bin/env python
+"""Bench of the SQAP-VLA hot path on B200: W4A4 linears of a Llama-2-7B-style layer on a batch of
+observations, with the quantization-aware visual-token pruning between two layers.
+
+One step (per rank, 16 observations x 288 token rows = 4608 rows, configuration 4 of the workload):
+  layer A at M = 4608 : quantize(+Hadamard) -> QKV -> quantize -> O -> quantize -> gate/up (SwiGLU) -> quantize -> down
+  prune               : scores -> top-k U ring U FPS -> compaction -> row gather   (256 -> 128 visual tokens)
+  layer B at M = 2560 : the same four linears on the surviving rows (distinct weights)
+  decode              : one new token per observation (M = 16) through layer B's linears
+`value` = algorithmic tera-ops (2*M*N*K of every linear) per second of whole-step time, all ranks.
+
+Usage: python bench.py [--gpus N] [--steps K] [--warmup W] [--impl ours|reference]
+"""
+from __future__ import annotations
+
+import argparse
+import json
+import os
+import subprocess
+import sys
+import threading
+import time
+
+import numpy as np
+
+ROOT = os.path.dirname(os.path.abspath(__file__))
+sys.path.insert(0, ROOT)
+
+from paper_2509_09090_b200 import workloads as wl  # noqa: E402
+from paper_2509_09090_b200 import dist_utils as du  # noqa: E402
+
+N_OBS = 16
+KEEP = 128
+K_ATTN = 64
+RING_RADIUS = 1
+M_FULL = N_OBS * wl.ROWS
+ROWS_KEPT = 32 + KEEP
+M_PRUNED = N_OBS * ROWS_KEPT
+METRIC = "W4A4 linear TOPS (whole pruned-prefill step); tokens/s beside it"
+WORKLOAD = ("configs[4]: 16 observations x 288 tokens (4608 rows), Llama-2-7B QKV/O/gate-up/down W4A4, "
+            "prune 256->128 visual tokens (top-k 64 U ring R_t=1 U FPS), pruned layer at 2560 rows, decode at 16 rows")
+
+
+def layer_ops(M: int) -> float:
+    H, F = wl.HIDDEN, wl.FFN
+    return 2.0 * M * (H * 3 * H + H * H + 2 * H * F + F * H)
+
+
+STEP_OPS = layer_ops(M_FULL) + layer_ops(M_PRUNED) + layer_ops(N_OBS)
+
+
+def measured_peaks():
+    path = os.path.join(ROOT, "MEASURED_PEAKS.json")
+    if os.path.exists(path):
+        with open(path) as fh:
+            d = json.load(fh)
+        return dict(hbm_gbs=d["hbm_gbs"], bf16=d["bf16_tflops"], bf16_sustained=d["bf16_tflops_sustained"],
+                    source="measured")
+    return dict(hbm_gbs=6650.0, bf16=1590.0, bf16_sustained=1400.0, source="fallback")
+
+
+# ----------------------------------------------------------------------------------------- clocks
+
+class ClockSampler:
+    """Samples nvidia-smi clocks and throttle reasons while the timed region runs."""
+    Q = ("index,clocks.sm,clocks.max.sm,power.draw,clocks_event_reasons.active,clocks_event_reasons.hw_slowdown,"
+         "clocks_event_reasons.hw_thermal_slowdown,clocks_event_reasons.sw_thermal_slowdown,"
+         "clocks_event_reasons.sw_power_cap")
+
+    def __init__(self, gpu_index: int):
+        self.gpu_index, self.proc, self.lines = gpu_index, None, []
+
+    def start(self):
+        try:
+            self.proc = subprocess.Popen(["nvidia-smi", f"--query-gpu={self.Q}", "--format=csv,noheader,nounits",
+                                          "-lms", "100", "-i", str(self.gpu_index)], stdout=subprocess.PIPE,
+                                         stderr=subprocess.DEVNULL, text=True)
+            self.thread = threading.Thread(target=self._read, daemon=True)
+            self.thread.start()
+        except Exception:
+            self.proc = None
+
+    def _read(self):
+        for line in self.proc.stdout:
+            self.lines.append(line.strip())
+
+    def stop(self) -> dict:
+        if self.proc is None:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["nvidia-smi unavailable"])
+        time.sleep(0.15)
+        self.proc.terminate()
+        try:
+            self.proc.wait(timeout=2)
+        except Exception:
+            self.proc.kill()
+        sm, mx, reasons = [], [], set()
+        names = ["hw_slowdown", "hw_thermal_slowdown", "sw_thermal_slowdown", "sw_power_cap"]
+        for ln in self.lines:
+            f = [t.strip() for t in ln.split(",")]
+            if len(f) < 9:
+                continue
+            try:
+                sm.append(float(f[1]))
+                mx.append(float(f[2]))
+            except ValueError:
+                continue
+            for nm, val in zip(names, f[5:9]):
+                if val.lower().startswith("active"):
+                    reasons.add(nm)
+        if not sm:
+            return dict(sm_mhz=None, sm_max_mhz=None, reasons=["no samples"])
+        return dict(sm_mhz=float(np.median(sm)), sm_max_mhz=float(np.max(mx)), reasons=sorted(reasons),
+                    samples=len(sm))
+
+
+# ----------------------------------------------------------------------------------------- our arm
+
+class Layer:
+    def __init__(self, B, G_pack, weights: dict):
+        self.w = {}
+        for name, N, K in wl.LAYER_LINEARS:
+            self.w[name] = G_pack(weights[name + "_codes"], weights[name + "_scales"], N, K)
+
+
+class Path:
+    """Device state of one rank and the step function (all work goes through the C ABI)."""
+
+    def __init__(self, torch, B, device, seed: int):
+        self.torch, self.B, self.dev = torch, B, device
+        t = torch
+        inp = wl.config4_inputs(seed=seed, batch=N_OBS)
+        self.x_host = t.from_numpy(inp["x"].reshape(M_FULL, wl.HIDDEN)).pin_memory()
+        self.scores_host = t.from_numpy(inp["scores"]).pin_memory()
+        self.centers_host = t.from_numpy(inp["centers"]).pin_memory()
+        self.xdec_host = t.from_numpy(wl.activations(seed, wl.T_X2, N_OBS, wl.HIDDEN, 41, 30.0)).pin_memory()
+        on_dev = lambda h: t.empty(h.shape, dtype=h.dtype, device=device)
+        self.x, self.scores = on_dev(self.x_host), on_dev(self.scores_host)
+        self.centers, self.xdec = on_dev(self.centers_host), on_dev(self.xdec_host)
+
+        def pack(codes, scales, N, K):
+            return B.sqap_pack_weights(np.ascontiguousarray(codes), np.ascontiguousarray(scales), N, K)
+
+        self.layers = []
+        for li in range(2):
+            wts = wl.config4_weights(seed=seed + 100 * li)
+            self.layers.append(Layer(B, pack, wts))
+            del wts
+        M = M_FULL
+        f16, u8, f32, i32 = t.float16, t.uint8, t.float32, t.int32
+        self.q = t.empty(M * wl.FFN // 2, dtype=u8, device=device)
+        self.sx = t.empty(M, dtype=f32, device=device)
+        self.qkv = t.empty(M, wl.QKV, dtype=f16, device=device)
+        self.o = t.empty(M, wl.HIDDEN, dtype=f16, device=device)
+        self.h = t.empty(M, wl.FFN, dtype=f16, device=device)
+        self.d = t.empty(M, wl.HIDDEN, dtype=f16, device=device)
+        self.x1 = t.empty(M_PRUNED, wl.HIDDEN, dtype=f16, device=device)
+        self.d1 = t.empty(M_PRUNED, wl.HIDDEN, dtype=f16, device=device)
+        self.ddec = t.empty(N_OBS, wl.HIDDEN, dtype=f16, device=device)
+        self.kept = t.empty(N_OBS, wl.ROWS, dtype=i32, device=device)
+        self.nkept = t.empty(N_OBS, dtype=i32, device=device)
+        self.ws_bytes = B.sqap_workspace_bytes(M, wl.QKV, wl.FFN)
+        self.ws = t.empty(self.ws_bytes, dtype=u8, device=device)
+        assert self.ws.data_ptr() % 256 == 0
+        self.prune_params = wl.prune_params(N_OBS, wl.ROWS, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32,
+                                            K_ATTN, KEEP, ring_radius=RING_RADIUS)
+        self.d1_host = t.empty(M_PRUNED, wl.HIDDEN, dtype=f16).pin_memory()
+        self.ddec_host = t.empty(N_OBS, wl.HIDDEN, dtype=f16).pin_memory()
+        self.kept_host = t.empty(N_OBS, wl.ROWS, dtype=i32).pin_memory()
+        self.h2d_bytes = sum(v.numel() * v.element_size() for v in
+                             (self.x_host, self.scores_host, self.centers_host, self.xdec_host))
+        self.d2h_bytes = sum(v.numel() * v.element_size() for v in (self.d1_host, self.ddec_host, self.kept_host))
+        self.gemm_events = []
+
+    def linear(self, x_ptr, M, K, ldx, w, w_up, out, rotate=False, flags=0):
+        B = self.B
+        B.sqap_quantize_act(x_ptr, M, K, ldx, None, B.SQAP_Q_ROTATE if rotate else 0, self.q, self.sx)
+        B.sqap_w4a4_linear(self.q, self.sx, M, w, w_up, out, out.shape[1], B.SQAP_FP16, flags, self.ws, self.ws_bytes)
+
+    def layer(self, x, M, L: Layer, d_out):
+        H = wl.HIDDEN
+        self.linear(x.data_ptr(), M, H, H, L.w["qkv"], None, self.qkv, rotate=True)
+        self.linear(self.qkv.data_ptr() + 2 * 2 * H, M, H, wl.QKV, L.w["o"], None, self.o)   # V third of QKV
+        self.linear(self.o.data_ptr(), M, H, H, L.w["gate"], L.w["up"], self.h)
+        self.linear(self.h.data_ptr(), M, wl.FFN, wl.FFN, L.w["down"], None, d_out)
+
+    def step(self):
+        B = self.B
+        self.layer(self.x, M_FULL, self.layers[0], self.d)
+        B.sqap_prune_tokens(self.prune_params, self.scores, self.centers, self.x, wl.HIDDEN, wl.HIDDEN, self.x1,
+                            wl.HIDDEN, ROWS_KEPT, self.kept, self.nkept)
+        self.layer(self.x1, M_PRUNED, self.layers[1], self.d1)
+        self.layer(self.xdec, N_OBS, self.layers[1], self.ddec)
+
+    def upload(self):
+        self.x.copy_(self.x_host, non_blocking=True)
+        self.scores.copy_(self.scores_host, non_blocking=True)
+        self.centers.copy_(self.centers_host, non_blocking=True)
+        self.xdec.copy_(self.xdec_host, non_blocking=True)
+
+    def download(self):
+        self.d1_host.copy_(self.d1, non_blocking=True)
+        self.ddec_host.copy_(self.ddec, non_blocking=True)
+        self.kept_host.copy_(self.kept, non_blocking=True)
+
+
+def time_region(torch, fn, steps: int, world: int):
+    du.barrier(world)
+    torch.cuda.synchronize()
+    e0, e1 = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+    e0.record()
+    for _ in range(steps):
+        fn()
+    e1.record()
+    torch.cuda.synchronize()
+    du.barrier(world)
+    ms = e0.elapsed_time(e1)
+    return du.max_over_ranks(ms, world, device="cuda")
+
+
+def dominant_gemm_roofline(torch, B, path: Path, steps: int, peaks: dict):
+    """The QKV GEMM at M = 4608 (largest single launch), timed alone with CUDA events on its stream.
+    The expand pass is skipped (SQAP_L_REUSE_EXPANDED), so the events bracket exactly one GEMM launch."""
+    L0, L1 = path.layers
+    M, N, K = M_FULL, wl.QKV, wl.HIDDEN
+    B.sqap_quantize_act(path.x, M, K, K, None, B.SQAP_Q_ROTATE, path.q, path.sx)
+    B.sqap_w4a4_linear(path.q, path.sx, M, L0.w["qkv"], None, path.qkv, N, B.SQAP_FP16, 0, path.ws, path.ws_bytes)
+    ws = [L0.w["qkv"], L1.w["qkv"]]
+    for i in range(3):
+        B.sqap_w4a4_linear(path.q, path.sx, M, ws[i % 2], None, path.qkv, N, B.SQAP_FP16, B.SQAP_L_REUSE_EXPANDED,
+                           path.ws, path.ws_bytes)
+    torch.cuda.synchronize()
+    evs = []
+    for i in range(steps):
+        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+        a.record()
+        B.sqap_w4a4_linear(path.q, path.sx, M, ws[i % 2], None, path.qkv, N, B.SQAP_FP16, B.SQAP_L_REUSE_EXPANDED,
+                           path.ws, path.ws_bytes)
+        b.record()
+        evs.append((a, b))
+    torch.cuda.synchronize()
+    ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    ops = 2.0 * M * N * K
+    achieved = ops / (ms * 1e-3) / 1e12
+    peak = 2.0 * peaks["bf16"]       # int8 dense = 2 x bf16 dense (nominal ratio) x the measured bf16 burst figure
+    return dict(bound="tensor", kernel="w4a4 linear GEMM, M=4608 N=12288 K=4096 (int8 MMA, int32 accumulate)",
+                achieved=achieved, peak=peak, unit="TOP/s", frac=achieved / peak, traffic=None,
+                peak_source=f"2 x bf16 burst ({peaks['source']})", ms_per_launch=ms)
+
+
+def cpu_baseline(seconds_budget: float = 20.0):
+    """The oracle, as it stands, on the host cores: a bounded sample of the same step (rows of one
+    observation through layer A's linears plus the pruning criterion of that observation)."""
+    import oracle
+    oracle.build()
+    wts = wl.config4_weights(seed=4)
+    x = wl.config4_inputs(seed=4, batch=1)
+    rows = 8
+    xs = x["x"][0, :rows]
+    t0 = time.perf_counter()
+    _oracle_layer(oracle, xs, wts)
+    dt = time.perf_counter() - t0
+    rows = int(max(8, min(wl.ROWS, rows * seconds_budget / max(dt, 1e-3) * 0.8)))
+    xs = x["x"][0, :rows]
+    t0 = time.perf_counter()
+    _oracle_layer(oracle, xs, wts)
+    p = wl.prune_params(1, wl.ROWS, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32, K_ATTN, KEEP,
+                        ring_radius=RING_RADIUS)
+    oracle.prune_tokens(p, x["scores"].view(np.uint16), x["centers"])
+    dt = time.perf_counter() - t0
+    ops = layer_ops(rows)
+    return dict(value=ops / dt / 1e12, unit="TOPS", cores=oracle.num_threads(), kind="oracle",
+                sample=f"{rows} token rows of one observation through one layer's four W4A4 linears + the pruning "
+                       f"criterion of that observation ({dt:.1f} s)", tokens_per_s=rows / dt)
+
+
+def _oracle_layer(oracle, x_f16, wts):
+    def lin(xin, name, rotate=False, up=None):
+        _, s, codes = oracle.quantize_act(np.ascontiguousarray(xin).view(np.uint16), rotate=rotate)
+        acc = oracle.gemm_i32(codes, wts[name + "_codes"])
+        sw = wts[name + "_scales"].view(np.uint16)
+        if up is None:
+            return oracle.epilogue(acc, s, sw).view(np.float16)
+        acc_u = oracle.gemm_i32(codes, wts[up + "_codes"])
+        return oracle.epilogue_swiglu(acc, acc_u, s, sw, wts[up + "_scales"].view(np.uint16)).view(np.float16)
+
+    qkv = lin(x_f16, "qkv", rotate=True)
+    o = lin(qkv[:, 2 * wl.HIDDEN:], "o")
+    h = lin(o, "gate", up="up")
+    return lin(h, "down")
+
+
+def run_ours(args):
+    import torch
+    from paper_2509_09090_b200 import binding as B
+    if not torch.cuda.is_available():
+        raise SystemExit("bench.py: no CUDA device; the product path has no CPU fallback")
+    rank, local_rank, world = du.init("nccl") if args.gpus > 1 else (0, 0, 1)
+    torch.cuda.set_device(local_rank)
+    device = torch.device("cuda", local_rank)
+    B.lib()
+    peaks = measured_peaks()
+    path = Path(torch, B, device, seed=4 + 1000 * rank)
+    path.upload()
+    torch.cuda.synchronize()
+
+    for _ in range(max(args.warmup, 3)):
+        path.step()
+    torch.cuda.synchronize()
+    if B.sqap_device_status() != B.SQAP_OK:
+        raise SystemExit("bench.py: a kernel reported an expired bounded wait")
+
+    sampler = ClockSampler(local_rank)
+    if rank == 0:
+        sampler.start()
+    l0 = B.sqap_kernel_launch_count()
+    ms = time_region(torch, path.step, args.steps, world)
+    launches = B.sqap_kernel_launch_count() - l0
+    clocks = sampler.stop() if rank == 0 else None
+
+    def e2e_step():
+        path.upload()
+        path.step()
+        path.download()
+
+    for _ in range(2):
+        e2e_step()
+    ms_e2e = time_region(torch, e2e_step, args.steps, world)
+    roof = dominant_gemm_roofline(torch, B, path, max(args.steps, 10), peaks) if rank == 0 else None
+    if B.sqap_device_status() != B.SQAP_OK:
+        raise SystemExit("bench.py: a kernel reported an expired bounded wait")
+
+    ms_step = ms / args.steps
+    tops = world * STEP_OPS / (ms_step * 1e-3) / 1e12
+    tops_e2e = world * STEP_OPS / (ms_e2e / args.steps * 1e-3) / 1e12
+    if rank == 0:
+        cpu = cpu_baseline() if world == 1 and not args.no_cpu_baseline else None
+        line = {
+            "metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": world, "steps": args.steps,
+            "warmup": max(args.warmup, 3), "ms_per_step": ms_step, "higher_is_better": True, "scaling": "weak",
+            "vs_baseline": None, "dtype": "int8 x int8 -> int32 (INT4 codes), fp32 epilogue, fp16 out",
+            "data": "synthetic",
+            "config": {"workload": WORKLOAD, "observations_per_gpu": N_OBS, "rows_per_observation": wl.ROWS,
+                       "keep_visual": KEEP, "l2": "inputs larger than L2 (202 MB packed weights, 38 MB activations, "
+                                                  "113 MB QKV output per step)"},
+            "tokens_per_s": world * M_FULL / (ms_step * 1e-3),
+            "e2e": {"value": tops_e2e, "unit": "TOPS", "h2d_bytes_per_step": path.h2d_bytes,
+                    "d2h_bytes_per_step": path.d2h_bytes, "tokens_per_s": world * M_FULL / (ms_e2e / args.steps * 1e-3)},
+            "gpu_launches": int(launches),
+            "clocks": clocks,
+            "roofline": roof,
+            "cpu_baseline": cpu,
+        }
+        print(json.dumps(line))
+    du.finish(world)
+
+
+def run_reference(args):
+    """The reference arm is the CPU oracle, timed on the host cores (rank 0 only)."""
+    rank, _, world = du.world_from_env()
+    if rank != 0:
+        return
+    import oracle
+    oracle.build()
+    wts = wl.config4_weights(seed=4)
+    x = wl.config4_inputs(seed=4, batch=1)
+    p = wl.prune_params(1, wl.ROWS, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32, K_ATTN, KEEP,
+                        ring_radius=RING_RADIUS)
+    t0 = time.perf_counter()
+    _oracle_layer(oracle, x["x"][0, :4], wts)
+    per_row = (time.perf_counter() - t0) / 4
+    total = args.steps + args.warmup
+    rows = int(max(1, min(wl.ROWS, 150.0 / max(total, 1) / max(per_row, 1e-4))))
+
+    def step():
+        _oracle_layer(oracle, x["x"][0, :rows], wts)
+        oracle.prune_tokens(p, x["scores"].view(np.uint16), x["centers"])
+
+    for _ in range(args.warmup):
+        step()
+    t0 = time.perf_counter()
+    for _ in range(args.steps):
+        step()
+    dt = (time.perf_counter() - t0) / max(args.steps, 1)
+    tops = layer_ops(rows) / dt / 1e12
+    sample = (f"{rows} token rows of one observation through one layer's four W4A4 linears + the pruning criterion "
+              f"of that observation, per step")
+    print(json.dumps({
+        "impl": "reference", "metric": METRIC, "value": tops, "unit": "TOPS", "n_gpus": args.gpus,
+        "steps": args.steps, "warmup": args.warmup, "ms_per_step": dt * 1e3, "higher_is_better": True,
+        "scaling": "weak", "vs_baseline": None, "dtype": "int32 exact / fp32 (CPU oracle)", "data": "synthetic",
+        "config": {"workload": WORKLOAD, "sample": sample},
+        "tokens_per_s": rows / dt,
+        "cpu_baseline": {"value": tops, "unit": "TOPS", "cores": oracle.num_threads(), "kind": "oracle",
+                         "sample": sample},
+        "e2e": {"value": tops, "unit": "TOPS", "h2d_bytes_per_step": 0, "d2h_bytes_per_step": 0},
+    }))
+
+
+def main():
+    ap = argparse.ArgumentParser()
+    ap.add_argument("--gpus", type=int, default=1)
+    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--warmup", type=int, default=3)
+    ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
+    ap.add_argument("--no-cpu-baseline", action="store_true")
+    args = ap.parse_args()
+    if args.impl == "reference":
+        run_reference(args)
+    else:
+        run_ours(args)
+
+
+if __name__ == "__main__":
+    main()

@@ -1,0 +1,186 @@
+/*
+ * sqap.h — C ABI of the SQAP-VLA hot path for NVIDIA B200 (sm_100a).
+ *
+ * The path is the part of a W4A4 vision-language-action model that the paper speeds up:
+ * the 4-bit-weight / 4-bit-activation linear layers of the language backbone, run on a
+ * visual-token set reduced by the paper's quantization-aware pruning criterion
+ * (K_final = K_attn U K_ring U K_fps).
+ *
+ * General rules for every call
+ *   - "device" pointers are CUDA device pointers owned by the CALLER; the library never
+ *     frees or keeps them. "host" pointers are ordinary host memory.
+ *   - `stream` is a cudaStream_t passed as void* (NULL = the legacy default stream). Calls
+ *     validate their arguments on the host, enqueue work on `stream` and return without
+ *     synchronising, unless stated otherwise.
+ *   - Sizes are `int`, row strides `int64_t`, both counted in ELEMENTS of the array's type.
+ *   - Return value is a sqap_status; nothing throws, aborts or prints. Nothing runs on the CPU
+ *     in place of a kernel: without a usable sm_100 device the compute calls fail.
+ *   - Inputs must be finite. Non-finite activations or scores give unspecified codes /
+ *     indices, never a fault.
+ */
+#ifndef SQAP_H
+#define SQAP_H
+
+#include <stddef.h>
+#include <stdint.h>
+
+#ifdef __cplusplus
+extern "C" {
+#endif
+
+typedef enum {
+    SQAP_OK = 0,
+    SQAP_ERR_INVALID = 1,     /* null pointer, negative or inconsistent size */
+    SQAP_ERR_RANGE = 2,       /* weight code outside [-8,7]; scale not finite or <= 0 */
+    SQAP_ERR_ALIGN = 3,       /* pointer or stride not 16-byte aligned; K not a multiple of 32 */
+    SQAP_ERR_UNSUPPORTED = 4, /* e.g. rotation with K not a power of two; n_visual > 1024 */
+    SQAP_ERR_NOMEM = 5,       /* device allocation failed, or workspace too small */
+    SQAP_ERR_CUDA = 6,        /* a CUDA call failed; see sqap_last_cuda_error() */
+    SQAP_ERR_TIMEOUT = 7      /* a bounded wait inside a kernel ran out (reported by sqap_device_status) */
+} sqap_status;
+
+/* Output element types of sqap_w4a4_linear. */
+#define SQAP_FP16 0
+#define SQAP_BF16 1
+#define SQAP_I32 2 /* raw int32 accumulators (checking only; SwiGLU not allowed) */
+
+/* Flags of sqap_quantize_act. */
+#define SQAP_Q_ROTATE 1u /* apply the orthonormal Hadamard rotation to each row first (Eq. 6) */
+
+/* Flags of sqap_pack_weights. */
+#define SQAP_W_ROTATED 1u /* bookkeeping only: the codes are those of W·H^T (Eq. 6, weight side) */
+
+/* Flags of sqap_w4a4_linear (0 = let the library choose the kernel). */
+#define SQAP_L_FORCE_SIMT 1u    /* the plain CUDA-core kernel */
+#define SQAP_L_FORCE_TCGEN05 2u /* the tcgen05 tensor-core kernel (needs K % 128 == 0) */
+#define SQAP_L_FORCE_GEMV 4u    /* the weight-streaming kernel for very few rows (M <= 8) */
+#define SQAP_L_REUSE_EXPANDED 8u /* the workspace still holds the expanded form of these same M x K activations
+                                    from the previous call that used it (one activation feeding several weight
+                                    matrices): skip the expand pass */
+
+/* Opaque packed weight matrix; owned by the LIBRARY, released by sqap_free_weights. Immutable
+ * after creation and usable from any stream once the creating stream has reached the pack. */
+typedef struct sqap_weights sqap_weights;
+
+/*
+ * Offline weight side of W4A4 ("4-bit weights", introduction; Eq. 6 for rotated layers):
+ * takes INT4 codes [N rows = output channels][K] (row-major, one int8 per code, values -8..7)
+ * and one fp16 scale per output channel (bits as uint16, finite, > 0) and stores them in the
+ * library's private nibble-packed device layout (N*K/2 bytes + 2N bytes of scales). `codes` and `scales_fp16` may each be host or device memory. The call allocates
+ * device memory, synchronises `stream` before returning (it validates the codes), and writes the
+ * handle to *out. Errors: INVALID (null, N <= 0, K <= 0), ALIGN (K % 32), RANGE, NOMEM, CUDA.
+ */
+sqap_status sqap_pack_weights(const int8_t* codes, const uint16_t* scales_fp16, int N, int K, uint32_t flags,
+                              void* stream, sqap_weights** out);
+
+/* Releases a handle (NULL is accepted). Synchronises the device. */
+sqap_status sqap_free_weights(sqap_weights* w);
+
+/* Shape and flags of a handle. */
+sqap_status sqap_weights_info(const sqap_weights* w, int* N, int* K, uint32_t* flags);
+
+/* Inverse of the packing, for checking: writes the original codes [N*K] and scale bits [N] to
+ * HOST memory. Synchronises. */
+sqap_status sqap_unpack_weights(const sqap_weights* w, int8_t* codes_out_host, uint16_t* scales_out_host);
+
+/*
+ * Online activation side of W4A4 ("4-bit activations"; Section "Pruning-Targeted Quantizer
+ * Enhancement"): per-token symmetric INT4 quantization of fp16 rows.
+ *   v = fp32(x[row])                    ; with SQAP_Q_ROTATE: v = H v, H = Sylvester-Hadamard / sqrt(K)
+ *   amax = max|v| ; scale = amax / 7 (1 if the row is all zero) ; inv = 7 / amax
+ *   q = clamp(round_half_even(v * inv), -8, 7)
+ * x: device fp16, row i starts at x + src*ldx with src = row_index ? row_index[i] : i.
+ * row_index: device int32 [M] or NULL. K % 32 == 0; ROTATE needs K a power of two, 64 <= K <= 16384.
+ * q_packed: device [M][K/2] bytes, PUBLIC layout: byte j of a row = (q[2j] & 15) | (q[2j+1] & 15) << 4
+ * (two's-complement nibbles). scales: device fp32 [M]. M = 0 is a no-op.
+ * x, q_packed 16-byte aligned; ldx % 8 == 0.
+ */
+sqap_status sqap_quantize_act(const void* x, int M, int K, int64_t ldx, const int32_t* row_index, uint32_t flags,
+                              uint8_t* q_packed, float* scales, void* stream);
+
+/* Bytes of caller-provided scratch that sqap_w4a4_linear needs for M rows against a K-column
+ * weight matrix (independent of N). Always a multiple of 256. */
+size_t sqap_workspace_bytes(int M, int N, int K, uint32_t flags);
+
+/*
+ * The W4A4 linear (Q = W_q^T X on integer codes, then dequantisation):
+ *   acc[m][n] = sum_k q[m][k] * w[n][k]                       exact int32
+ *   out[m][n] = round( (float(acc) * act_scales[m]) * float(w_scale[n]) )       fp16 or bf16
+ * With w_up != NULL (the gated MLP; w = gate projection, same N and K):
+ *   g, u as above in fp32 from w and w_up;  out = round( g / (1 + exp(-g)) * u )
+ * q_packed / act_scales: device, as written by sqap_quantize_act (K = the handle's K).
+ * out: device [M rows, ldo elements apart] of out_dtype; 16-byte aligned, ldo*elemsize % 16 == 0.
+ * workspace: device scratch of at least sqap_workspace_bytes(M, N, K, flags) bytes, 256-byte
+ * aligned; its contents are undefined afterwards; two calls in flight at once need two workspaces.
+ * flags: SQAP_L_* or 0 (at most one FORCE flag). Errors: INVALID, ALIGN, UNSUPPORTED (forced kernel cannot run the shape),
+ * NOMEM (workspace too small), CUDA.
+ */
+sqap_status sqap_w4a4_linear(const uint8_t* q_packed, const float* act_scales, int M, const sqap_weights* w,
+                             const sqap_weights* w_up, void* out, int64_t ldo, int out_dtype, uint32_t flags,
+                             void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * Parameters of the pruning criterion (Section "Quantization-aware Pruning Strategies").
+ * An observation is `rows` consecutive token rows; rows [visual_start, visual_start + n_visual)
+ * are the visual tokens, laid out row-major on a grid_w x grid_h token grid
+ * (token j has t_u = j % grid_w, t_v = j / grid_w); all other rows are never pruned.
+ */
+typedef struct {
+    int batch;        /* observations */
+    int rows;         /* token rows per observation */
+    int visual_start; /* first visual row */
+    int n_visual;     /* N_v = grid_w * grid_h, at most 1024 */
+    int grid_w, grid_h;
+    int score_rows;  /* R > 0: scores are fp16 [batch][R][n_visual], summed over R in fp32, row 0 first;
+                        R = 0: scores are fp32 [batch][n_visual] */
+    int k_attn;      /* |K_attn|: tokens kept for their score (Eq. 1); ties -> lower index */
+    int keep_total;  /* visual tokens to keep in all; FPS fills keep_total - |K_attn U K_ring| */
+    int ring_radius; /* R_t of Eq. 4; < 0: no ring */
+    uint32_t flags;  /* 0 */
+} sqap_prune_params;
+
+/*
+ * Quantization-aware visual-token pruning and compaction.
+ *   K_attn = the k_attn highest-scoring visual tokens                                  (Eq. 1)
+ *   K_ring = tokens within Chebyshev distance ring_radius of ring_center                (Eq. 4)
+ *   K_fps  = farthest-point sampling of the quota's remainder from the other tokens     (Eq. 5)
+ *            (squared Euclidean grid distance; first pick = lowest remaining index; ties -> lower index)
+ *   kept rows = all non-visual rows + visual_start + j for j in K_attn U K_ring U K_fps, ascending.
+ * scores: device (see score_rows). ring_center: device int32 [batch][2] = (t_u, t_v), may lie off the
+ * grid; NULL or ring_radius < 0 disables the ring. x: device fp16 [batch*rows rows, ldx apart], or NULL
+ * for indices only; x_out: device fp16, observation b's kept rows are written contiguously starting at
+ * row b*out_rows (ldo apart), in ascending original order — the caller guarantees n_kept <= out_rows
+ * (rows beyond out_rows are dropped, never written). kept_idx: device int32 [batch][rows], first
+ * n_kept[b] entries valid (row numbers within the observation), the rest -1. n_kept: device int32 [batch].
+ * K % 8 == 0; x, x_out 16-byte aligned; ldx, ldo % 8 == 0.
+ */
+sqap_status sqap_prune_tokens(const sqap_prune_params* p, const void* scores, const int32_t* ring_center,
+                              const void* x, int64_t ldx, int K, void* x_out, int64_t ldo, int out_rows,
+                              int32_t* kept_idx, int32_t* n_kept, void* stream);
+
+/*
+ * Host helper (no GPU): robot-aware protection, Eq. 2-3. Projects the world point xyz through the
+ * intrinsics Kmat (3x3 row-major) and extrinsics Rt = [R|t] (3x4 row-major) and maps the pixel to
+ * token coordinates with the patch size (patch_w, patch_h), in double precision:
+ * t_u = floor(u / patch_w), t_v = floor(v / patch_h). *in_front = 0 when the point is not in front
+ * of the camera (lambda <= 0); the coordinates are then 0 and no ring should be used.
+ */
+sqap_status sqap_project_center(const double Kmat[9], const double Rt[12], const double xyz[3], double patch_w,
+                                double patch_h, int32_t out_tu_tv[2], int* in_front);
+
+/* Synchronises `stream`, then returns and clears the status word that kernels on the current
+ * device set when one of their bounded waits runs out (SQAP_ERR_TIMEOUT) — SQAP_OK otherwise. */
+sqap_status sqap_device_status(void* stream);
+
+/* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
+int sqap_last_cuda_error(void);
+
+const char* sqap_status_string(sqap_status s);
+
+/* Number of kernels this library has launched in this process (all threads). */
+int64_t sqap_kernel_launch_count(void);
+
+#ifdef __cplusplus
+}
+#endif
+#endif /* SQAP_H */

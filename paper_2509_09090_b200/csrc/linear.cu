@@ -1,0 +1,331 @@
+// W4A4 linear: dispatcher, the activation expand pass, the CUDA-core GEMM (any shape) and the
+// weight-streaming kernel for very few rows. The tensor-core kernel lives in linear_tc.cu.
+#include "linear.cuh"
+
+namespace sqap {
+
+// ---------------------------------------------------------------------------------------------
+// Expand pass: public nibble-packed activations -> int8 in the form the GEMM kernels multiply.
+// One CTA per row. A 16-byte packed chunk (32 codes) becomes 32 int8.
+__device__ __forceinline__ void expand_word(uint32_t w, bool times16, uint32_t& out0, uint32_t& out1) {
+    uint32_t e, o;  // byte b of e = code 2b, of o = code 2b+1
+    if (times16) {
+        e = (w << 4) & 0xF0F0F0F0u;
+        o = w & 0xF0F0F0F0u;
+    } else {
+        e = w & 0x0F0F0F0Fu;
+        o = (w >> 4) & 0x0F0F0F0Fu;
+        e |= (e & 0x08080808u) * 0x1Eu;  // sign-extend each nibble to a byte
+        o |= (o & 0x08080808u) * 0x1Eu;
+    }
+    out0 = __byte_perm(e, o, 0x5140);
+    out1 = __byte_perm(e, o, 0x7362);
+}
+
+__global__ void __launch_bounds__(128) expand_act_kernel(const uint8_t* __restrict__ q, int K, int half,
+                                                         int8_t* __restrict__ x8, int32_t* __restrict__ bias_sum) {
+    __shared__ int red[4];
+    const int row = blockIdx.x;
+    const uint4* src = reinterpret_cast<const uint4*>(q + static_cast<int64_t>(row) * (K / 2));
+    uint4* dst = reinterpret_cast<uint4*>(x8 + static_cast<int64_t>(row) * K);
+    int s16 = 0;
+    for (int c = threadIdx.x; c < K / 32; c += blockDim.x) {
+        const uint4 p = __ldg(src + c);
+        const uint32_t w[4] = {p.x, p.y, p.z, p.w};
+        uint32_t o[8];
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int k = c * 32 + i * 8;
+            const bool t16 = (k % (2 * half)) < half;
+            expand_word(w[i], t16, o[2 * i], o[2 * i + 1]);
+            if (t16) {
+                s16 = __dp4a(static_cast<int>(o[2 * i]), 0x01010101, s16);
+                s16 = __dp4a(static_cast<int>(o[2 * i + 1]), 0x01010101, s16);
+            }
+        }
+        dst[2 * c] = make_uint4(o[0], o[1], o[2], o[3]);
+        dst[2 * c + 1] = make_uint4(o[4], o[5], o[6], o[7]);
+    }
+#pragma unroll
+    for (int off = 16; off > 0; off >>= 1) s16 += __shfl_xor_sync(0xffffffffu, s16, off);
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = s16;
+    __syncthreads();
+    if (threadIdx.x == 0) bias_sum[row] = (red[0] + red[1] + red[2] + red[3]) >> 4;
+}
+
+// Offsets (in codes, relative to the start of the row) that the low / high nibbles of packed 16-byte
+// chunk c of a weight row cover.
+__device__ __forceinline__ void chunk_k(int c, int half, int& lo_k, int& hi_k) {
+    if (half == 64) {
+        lo_k = (c >> 2) * 128 + (c & 3) * 16;
+        hi_k = lo_k + 64;
+    } else {
+        lo_k = c * 32;
+        hi_k = lo_k + 16;
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// CUDA-core GEMM: 64x64 output tile per CTA, 128 codes of K per step, dp4a on int8 words held in
+// shared memory. Runs every shape the API accepts; the reference point for the other kernels.
+constexpr int ST_M = 64, ST_N = 64, ST_KW = 32;  // KW = 32-bit words of K per step
+
+template <bool SWIGLU>
+__global__ void __launch_bounds__(128) w4a4_simt_kernel(LinearArgs a) {
+    __shared__ uint32_t Xs[ST_M][ST_KW + 1];
+    __shared__ uint32_t Ws[ST_N][ST_KW + 1];
+    __shared__ uint32_t Us[SWIGLU ? ST_N : 1][ST_KW + 1];
+    const int tid = threadIdx.x;
+    const int tn = tid & 7, tm = tid >> 3;
+    const int m0 = blockIdx.y * ST_M, n0 = blockIdx.x * ST_N;
+    int acc[4][8], accu[SWIGLU ? 4 : 1][8];
+#pragma unroll
+    for (int i = 0; i < 4; ++i)
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            acc[i][j] = 0;
+            if (SWIGLU) accu[i][j] = 0;
+        }
+    const int chunks_per_row = a.K / 32;  // packed 16-byte chunks in a weight row
+    for (int k0 = 0; k0 < a.K; k0 += 128) {
+        // activations: 64 rows x 8 chunks of 16 int8
+        for (int i = tid; i < ST_M * 8; i += 128) {
+            const int r = i >> 3, c = i & 7;
+            uint4 v = make_uint4(0, 0, 0, 0);
+            if (m0 + r < a.M && k0 + c * 16 < a.K)
+                v = __ldg(reinterpret_cast<const uint4*>(a.x8 + static_cast<int64_t>(m0 + r) * a.K + k0) + c);
+            Xs[r][c * 4 + 0] = v.x;
+            Xs[r][c * 4 + 1] = v.y;
+            Xs[r][c * 4 + 2] = v.z;
+            Xs[r][c * 4 + 3] = v.w;
+        }
+        // weights: 64 rows x 4 packed chunks, masked into two int8 chunks each
+        for (int i = tid; i < ST_N * 4; i += 128) {
+            const int r = i >> 2, cl = i & 3;
+            const int c = k0 / 32 + cl;
+            int lo_k, hi_k;
+            chunk_k(c, a.half, lo_k, hi_k);
+            lo_k -= k0;
+            hi_k -= k0;
+            uint4 v = make_uint4(0, 0, 0, 0), u = make_uint4(0, 0, 0, 0);
+            const bool ok = (n0 + r < a.N) && (c < chunks_per_row);
+            if (ok) {
+                v = __ldg(reinterpret_cast<const uint4*>(a.w + static_cast<int64_t>(n0 + r) * (a.K / 2)) + c);
+                if (SWIGLU) u = __ldg(reinterpret_cast<const uint4*>(a.w_up + static_cast<int64_t>(n0 + r) * (a.K / 2)) + c);
+            }
+            if (lo_k >= 0 && hi_k + 16 <= 128) {  // always true for valid chunks; keeps indices provably in range
+                const uint32_t wv[4] = {v.x, v.y, v.z, v.w}, wu[4] = {u.x, u.y, u.z, u.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    Ws[r][lo_k / 4 + q] = wv[q] & 0x0F0F0F0Fu;
+                    Ws[r][hi_k / 4 + q] = wv[q] & 0xF0F0F0F0u;
+                    if (SWIGLU) {
+                        Us[r][lo_k / 4 + q] = wu[q] & 0x0F0F0F0Fu;
+                        Us[r][hi_k / 4 + q] = wu[q] & 0xF0F0F0F0u;
+                    }
+                }
+            }
+        }
+        __syncthreads();
+#pragma unroll 8
+        for (int kk = 0; kk < ST_KW; ++kk) {
+            int xa[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) xa[i] = static_cast<int>(Xs[tm * 4 + i][kk]);
+#pragma unroll
+            for (int j = 0; j < 8; ++j) {
+                const int wb = static_cast<int>(Ws[tn + 8 * j][kk]);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) acc[i][j] = __dp4a(xa[i], wb, acc[i][j]);
+                if (SWIGLU) {
+                    const int ub = static_cast<int>(Us[tn + 8 * j][kk]);
+#pragma unroll
+                    for (int i = 0; i < 4; ++i) accu[i][j] = __dp4a(xa[i], ub, accu[i][j]);
+                }
+            }
+        }
+        __syncthreads();
+    }
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const int m = m0 + tm * 4 + i;
+        if (m >= a.M) continue;
+        const int bs = a.bias_sum[m];
+        const float sx = a.act_scales[m];
+#pragma unroll
+        for (int j = 0; j < 8; ++j) {
+            const int n = n0 + tn + 8 * j;
+            if (n >= a.N) continue;
+            const int t = finish_acc(acc[i][j], bs);
+            float y = dequant(t, sx, __half2float(a.w_scales[n]));
+            if (SWIGLU) y = swiglu(y, dequant(finish_acc(accu[i][j], bs), sx, __half2float(a.w_up_scales[n])));
+            store_out(a.out, static_cast<int64_t>(m) * a.ldo + n, a.out_dtype, y, t);
+        }
+    }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Weight-streaming kernel for M <= 8 (the single-token decode steps): HBM-bound on the packed
+// weights, N*K/2 bytes per call. One warp owns one output channel and streams its row with
+// 128-bit loads; the few activation rows are re-read through L1.
+template <int MM, bool SWIGLU>
+__global__ void __launch_bounds__(256) w4a4_gemv_kernel(LinearArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int n = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5);
+    if (n >= a.N) return;
+    const uint4* wrow = reinterpret_cast<const uint4*>(a.w + static_cast<int64_t>(n) * (a.K / 2));
+    const uint4* urow = SWIGLU ? reinterpret_cast<const uint4*>(a.w_up + static_cast<int64_t>(n) * (a.K / 2)) : nullptr;
+    int acc[MM], accu[SWIGLU ? MM : 1];
+#pragma unroll
+    for (int m = 0; m < MM; ++m) {
+        acc[m] = 0;
+        if (SWIGLU) accu[m] = 0;
+    }
+    const int chunks = a.K / 32;
+#pragma unroll 4
+    for (int c = lane; c < chunks; c += 32) {
+        const uint4 wv = __ldg(wrow + c);
+        uint4 uv = make_uint4(0, 0, 0, 0);
+        if (SWIGLU) uv = __ldg(urow + c);
+        int lo_k, hi_k;
+        chunk_k(c, a.half, lo_k, hi_k);
+        const uint32_t w4[4] = {wv.x, wv.y, wv.z, wv.w}, u4[4] = {uv.x, uv.y, uv.z, uv.w};
+#pragma unroll
+        for (int m = 0; m < MM; ++m) {
+            if (m < a.M) {
+                const int8_t* xr = a.x8 + static_cast<int64_t>(m) * a.K;
+                const uint4 xl = __ldg(reinterpret_cast<const uint4*>(xr + lo_k));
+                const uint4 xh = __ldg(reinterpret_cast<const uint4*>(xr + hi_k));
+                const int l4[4] = {(int)xl.x, (int)xl.y, (int)xl.z, (int)xl.w};
+                const int h4[4] = {(int)xh.x, (int)xh.y, (int)xh.z, (int)xh.w};
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    acc[m] = __dp4a(l4[i], static_cast<int>(w4[i] & 0x0F0F0F0Fu), acc[m]);
+                    acc[m] = __dp4a(h4[i], static_cast<int>(w4[i] & 0xF0F0F0F0u), acc[m]);
+                    if (SWIGLU) {
+                        accu[m] = __dp4a(l4[i], static_cast<int>(u4[i] & 0x0F0F0F0Fu), accu[m]);
+                        accu[m] = __dp4a(h4[i], static_cast<int>(u4[i] & 0xF0F0F0F0u), accu[m]);
+                    }
+                }
+            }
+        }
+    }
+#pragma unroll
+    for (int m = 0; m < MM; ++m) {
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) {
+            acc[m] += __shfl_xor_sync(0xffffffffu, acc[m], off);
+            if (SWIGLU) accu[m] += __shfl_xor_sync(0xffffffffu, accu[m], off);
+        }
+    }
+    if (lane == 0) {
+        const float sw = __half2float(a.w_scales[n]);
+#pragma unroll
+        for (int m = 0; m < MM; ++m) {
+            if (m < a.M) {
+                const int bs = a.bias_sum[m];
+                const float sx = a.act_scales[m];
+                const int t = finish_acc(acc[m], bs);
+                float y = dequant(t, sx, sw);
+                if (SWIGLU) y = swiglu(y, dequant(finish_acc(accu[m], bs), sx, __half2float(a.w_up_scales[n])));
+                store_out(a.out, static_cast<int64_t>(m) * a.ldo + n, a.out_dtype, y, t);
+            }
+        }
+    }
+}
+
+template <int MM>
+static void launch_gemv(const LinearArgs& a, cudaStream_t s) {
+    const int warps = 8;
+    const int blocks = (a.N + warps - 1) / warps;
+    if (a.w_up) w4a4_gemv_kernel<MM, true><<<blocks, warps * 32, 0, s>>>(a);
+    else w4a4_gemv_kernel<MM, false><<<blocks, warps * 32, 0, s>>>(a);
+}
+
+static size_t round256(size_t v) { return (v + 255) / 256 * 256; }
+
+}  // namespace sqap
+
+extern "C" {
+
+size_t sqap_workspace_bytes(int M, int N, int K, uint32_t flags) {
+    (void)N;
+    (void)flags;
+    if (M <= 0 || K <= 0) return 256;
+    return sqap::round256(static_cast<size_t>(M) * K) + sqap::round256(sizeof(int32_t) * static_cast<size_t>(M));
+}
+
+sqap_status sqap_w4a4_linear(const uint8_t* q_packed, const float* act_scales, int M, const sqap_weights* w,
+                             const sqap_weights* w_up, void* out, int64_t ldo, int out_dtype, uint32_t flags,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+    using namespace sqap;
+    if (M < 0 || !w) return SQAP_ERR_INVALID;
+    if (out_dtype != SQAP_FP16 && out_dtype != SQAP_BF16 && out_dtype != SQAP_I32) return SQAP_ERR_INVALID;
+    if (flags & ~(SQAP_L_FORCE_SIMT | SQAP_L_FORCE_TCGEN05 | SQAP_L_FORCE_GEMV | SQAP_L_REUSE_EXPANDED))
+        return SQAP_ERR_INVALID;
+    const uint32_t force = flags & (SQAP_L_FORCE_SIMT | SQAP_L_FORCE_TCGEN05 | SQAP_L_FORCE_GEMV);
+    if ((force & (force - 1)) != 0) return SQAP_ERR_INVALID;  // at most one forced kernel
+    if (w_up && (w_up->N != w->N || w_up->K != w->K || w_up->half != w->half)) return SQAP_ERR_INVALID;
+    if (w_up && out_dtype == SQAP_I32) return SQAP_ERR_INVALID;
+    if (ldo < w->N) return SQAP_ERR_INVALID;
+    if (M == 0) return SQAP_OK;
+    if (!q_packed || !act_scales || !out || !workspace) return SQAP_ERR_INVALID;
+    const int esz = out_dtype == SQAP_I32 ? 4 : 2;
+    if (!aligned16(q_packed) || !aligned16(out) || (ldo * esz) % 16 != 0) return SQAP_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQAP_ERR_ALIGN;
+    if (workspace_bytes < sqap_workspace_bytes(M, w->N, w->K, flags)) return SQAP_ERR_NOMEM;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    LinearArgs a;
+    a.x8 = static_cast<int8_t*>(workspace);
+    a.bias_sum = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + round256(static_cast<size_t>(M) * w->K));
+    a.act_scales = act_scales;
+    a.M = M;
+    a.N = w->N;
+    a.K = w->K;
+    a.half = w->half;
+    a.w = w->packed;
+    a.w_scales = w->scales;
+    a.w_up = w_up ? w_up->packed : nullptr;
+    a.w_up_scales = w_up ? w_up->scales : nullptr;
+    a.out = out;
+    a.ldo = ldo;
+    a.out_dtype = out_dtype;
+
+    enum { SIMT, TC, GEMV } path;
+    if (flags & SQAP_L_FORCE_SIMT) path = SIMT;
+    else if (flags & SQAP_L_FORCE_GEMV) {
+        if (M > 8) return SQAP_ERR_UNSUPPORTED;
+        path = GEMV;
+    } else if (flags & SQAP_L_FORCE_TCGEN05) {
+        if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
+        path = TC;
+    } else {
+        path = M <= 8 ? GEMV : (tcgen05_supports(a) ? TC : SIMT);
+    }
+
+    sqap_status st = SQAP_OK;
+    if (!(flags & SQAP_L_REUSE_EXPANDED)) {
+        expand_act_kernel<<<M, 128, 0, s>>>(q_packed, a.K, a.half, const_cast<int8_t*>(a.x8),
+                                            const_cast<int32_t*>(a.bias_sum));
+        count_launch();
+        st = check_launch();
+        if (st != SQAP_OK) return st;
+    }
+
+    if (path == TC) return launch_linear_tcgen05(a, s);
+    if (path == GEMV) {
+        if (M == 1) launch_gemv<1>(a, s);
+        else if (M == 2) launch_gemv<2>(a, s);
+        else if (M <= 4) launch_gemv<4>(a, s);
+        else launch_gemv<8>(a, s);
+    } else {
+        dim3 grid((a.N + ST_N - 1) / ST_N, (M + ST_M - 1) / ST_M);
+        if (a.w_up) w4a4_simt_kernel<true><<<grid, 128, 0, s>>>(a);
+        else w4a4_simt_kernel<false><<<grid, 128, 0, s>>>(a);
+    }
+    count_launch();
+    return check_launch();
+}
+
+}  // extern "C"

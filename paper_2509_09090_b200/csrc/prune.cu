@@ -1,0 +1,183 @@
+// Quantization-aware visual-token pruning: K_final = K_attn U K_ring U K_fps, then compaction.
+//
+// One CTA per observation decides the kept set (a few KB of scores; latency-bound, the FPS loop
+// is m dependent steps), a second kernel copies the surviving rows (HBM-bound, 2 bytes read and
+// 2 written per kept element).
+#include "common.cuh"
+
+namespace sqap {
+
+constexpr int PRUNE_MAX_VISUAL = 1024;
+constexpr uint32_t FPS_D_INIT = 0x1FFFFFu;  // above any squared distance on a <= 1024-wide grid
+
+// CAND = visual tokens per lane of the FPS warp (token j lives in lane j % 32, slot j / 32).
+template <int CAND>
+__global__ void __launch_bounds__(512) prune_select_kernel(sqap_prune_params p, const void* __restrict__ scores,
+                                                            const int32_t* __restrict__ ring_center,
+                                                            int32_t* __restrict__ kept_idx,
+                                                            int32_t* __restrict__ n_kept) {
+    __shared__ float a[PRUNE_MAX_VISUAL];
+    __shared__ uint8_t keep[PRUNE_MAX_VISUAL];  // bit 0: in K_attn U K_ring, bit 1: in K_fps
+    __shared__ int warp_tot[32];
+    __shared__ int s_union;
+    const int b = blockIdx.x;
+    const int nv = p.n_visual;
+    const int tid = threadIdx.x, lane = tid & 31, warp = tid >> 5, nwarps = blockDim.x >> 5;
+
+    // scores: a_j = sum over the R score rows, row 0 first, in fp32
+    for (int j = tid; j < nv; j += blockDim.x) {
+        float s;
+        if (p.score_rows > 0) {
+            const __half* A = static_cast<const __half*>(scores) + static_cast<int64_t>(b) * p.score_rows * nv;
+            s = __half2float(A[j]);
+            for (int r = 1; r < p.score_rows; ++r) s = __fadd_rn(s, __half2float(A[static_cast<int64_t>(r) * nv + j]));
+        } else {
+            s = static_cast<const float*>(scores)[static_cast<int64_t>(b) * nv + j];
+        }
+        a[j] = s;
+    }
+    if (tid == 0) s_union = 0;
+    __syncthreads();
+
+    // Strategy 1 (Eq. 1): rank by counting under the order (score descending, index ascending).
+    // Strategy 2 (Eq. 4): Chebyshev ball around the projected robot position.
+    const bool ring_on = p.ring_radius >= 0 && ring_center != nullptr;
+    const int cu = ring_on ? ring_center[2 * b] : 0, cv = ring_on ? ring_center[2 * b + 1] : 0;
+    int local_union = 0;
+    for (int j = tid; j < nv; j += blockDim.x) {
+        const float aj = a[j];
+        int rank = 0;
+        for (int i = 0; i < nv; ++i) {
+            const float ai = a[i];
+            rank += (ai > aj) || (ai == aj && i < j);
+        }
+        bool in = rank < p.k_attn;
+        if (ring_on) {
+            const int du = abs(j % p.grid_w - cu), dv = abs(j / p.grid_w - cv);
+            in |= max(du, dv) <= p.ring_radius;
+        }
+        keep[j] = in ? 1 : 0;
+        local_union += in;
+    }
+    if (local_union) atomicAdd(&s_union, local_union);
+    __syncthreads();
+
+    // Strategy 3 (Eq. 5): farthest-point sampling by one warp. Key = D << 10 | (1023 - j): the
+    // maximum key is the largest distance, lowest index on ties; 0 marks "not a candidate".
+    const int m_fps = max(0, p.keep_total - s_union);
+    if (warp == 0 && m_fps > 0) {
+        uint32_t D[CAND];
+        int tu[CAND], tv[CAND];
+#pragma unroll
+        for (int i = 0; i < CAND; ++i) {
+            const int j = lane + 32 * i;
+            const bool cand = j < nv && keep[j] == 0;
+            D[i] = cand ? FPS_D_INIT : 0u;
+            tu[i] = j % p.grid_w;
+            tv[i] = j / p.grid_w;
+        }
+        for (int step = 0; step < m_fps; ++step) {
+            uint32_t best = 0;
+#pragma unroll
+            for (int i = 0; i < CAND; ++i) {
+                const uint32_t key = D[i] ? ((D[i] << 10) | static_cast<uint32_t>(1023 - (lane + 32 * i))) : 0u;
+                best = max(best, key);
+            }
+            best = __reduce_max_sync(0xffffffffu, best);
+            if (best == 0) break;  // remainder exhausted
+            const int pj = 1023 - static_cast<int>(best & 1023u);
+            const int pu = pj % p.grid_w, pv = pj / p.grid_w;
+            if ((pj & 31) == lane) keep[pj] = 2;
+#pragma unroll
+            for (int i = 0; i < CAND; ++i) {
+                const int du = tu[i] - pu, dv = tv[i] - pv;
+                const uint32_t d2 = static_cast<uint32_t>(du * du + dv * dv);  // 0 exactly for the picked token
+                D[i] = min(D[i], d2);
+            }
+        }
+    }
+    __syncthreads();
+
+    // Compaction: ascending row numbers of the kept rows (non-visual rows always kept).
+    int32_t* out = kept_idx + static_cast<int64_t>(b) * p.rows;
+    int base = 0;
+    for (int r0 = 0; r0 < p.rows; r0 += blockDim.x) {
+        const int r = r0 + tid;
+        bool k = false;
+        if (r < p.rows) {
+            const int j = r - p.visual_start;
+            k = (j < 0 || j >= nv) ? true : keep[j] != 0;
+        }
+        const uint32_t bal = __ballot_sync(0xffffffffu, k);
+        if (lane == 0) warp_tot[warp] = __popc(bal);
+        __syncthreads();
+        int before = 0, total = 0;
+        for (int w = 0; w < nwarps; ++w) {
+            const int t = warp_tot[w];
+            before += (w < warp) ? t : 0;
+            total += t;
+        }
+        if (k) out[base + before + __popc(bal & ((1u << lane) - 1u))] = r;
+        base += total;
+        __syncthreads();
+    }
+    for (int r = base + tid; r < p.rows; r += blockDim.x) out[r] = -1;
+    if (tid == 0) n_kept[b] = base;
+}
+
+// Row copy: grid (out_rows, batch); CTA (i, b) copies row kept_idx[b][i] of observation b.
+__global__ void __launch_bounds__(256) gather_rows_kernel(const __half* __restrict__ x, int64_t ldx, int rows, int K,
+                                                          const int32_t* __restrict__ kept_idx,
+                                                          const int32_t* __restrict__ n_kept, __half* __restrict__ out,
+                                                          int64_t ldo, int out_rows) {
+    const int i = blockIdx.x, b = blockIdx.y;
+    if (i >= n_kept[b]) return;
+    const int src = kept_idx[static_cast<int64_t>(b) * rows + i];
+    if (src < 0 || src >= rows) return;
+    const uint4* s = reinterpret_cast<const uint4*>(x + (static_cast<int64_t>(b) * rows + src) * ldx);
+    uint4* d = reinterpret_cast<uint4*>(out + (static_cast<int64_t>(b) * out_rows + i) * ldo);
+    for (int c = threadIdx.x; c < K / 8; c += blockDim.x) d[c] = __ldg(s + c);
+}
+
+}  // namespace sqap
+
+extern "C" sqap_status sqap_prune_tokens(const sqap_prune_params* p, const void* scores, const int32_t* ring_center,
+                                         const void* x, int64_t ldx, int K, void* x_out, int64_t ldo, int out_rows,
+                                         int32_t* kept_idx, int32_t* n_kept, void* stream) {
+    using namespace sqap;
+    if (!p) return SQAP_ERR_INVALID;
+    if (p->batch < 0 || p->rows < 0 || p->n_visual < 0 || p->visual_start < 0 ||
+        static_cast<int64_t>(p->visual_start) + p->n_visual > p->rows)
+        return SQAP_ERR_INVALID;
+    if (p->k_attn < 0 || p->keep_total < 0 || p->score_rows < 0 || p->flags != 0) return SQAP_ERR_INVALID;
+    if (p->n_visual > 0 && (p->grid_w <= 0 || p->grid_h <= 0 ||
+                            static_cast<int64_t>(p->grid_w) * p->grid_h != p->n_visual))
+        return SQAP_ERR_INVALID;
+    if (p->n_visual > PRUNE_MAX_VISUAL) return SQAP_ERR_UNSUPPORTED;
+    if (p->batch > 65535) return SQAP_ERR_UNSUPPORTED;
+    if (p->batch == 0) return SQAP_OK;
+    if (!kept_idx || !n_kept || (p->n_visual > 0 && !scores)) return SQAP_ERR_INVALID;
+    if (x) {
+        if (!x_out || K <= 0 || ldx < K || ldo < K || out_rows < 0) return SQAP_ERR_INVALID;
+        if (K % 8 != 0 || ldx % 8 != 0 || ldo % 8 != 0 || !aligned16(x) || !aligned16(x_out)) return SQAP_ERR_ALIGN;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    sqap_prune_params q = *p;
+    if (q.n_visual == 0) q.grid_w = q.grid_h = 1;
+    int threads = (q.n_visual + 31) / 32 * 32;
+    if (threads < 128) threads = 128;
+    if (threads > 512) threads = 512;
+    if (q.n_visual <= 256) prune_select_kernel<8><<<q.batch, threads, 0, s>>>(q, scores, ring_center, kept_idx, n_kept);
+    else prune_select_kernel<32><<<q.batch, threads, 0, s>>>(q, scores, ring_center, kept_idx, n_kept);
+    count_launch();
+    sqap_status st = check_launch();
+    if (st != SQAP_OK) return st;
+    if (x && out_rows > 0) {
+        dim3 grid(out_rows, q.batch);
+        gather_rows_kernel<<<grid, 256, 0, s>>>(static_cast<const __half*>(x), ldx, q.rows, K, kept_idx, n_kept,
+                                                static_cast<__half*>(x_out), ldo, out_rows);
+        count_launch();
+        st = check_launch();
+    }
+    return st;
+}

@@ -1,0 +1,409 @@
+"""Parity of the CUDA path (through the C ABI) with the CPU oracle on the same seeded inputs.
+
+Bar: INT4 codes, activation scales, int32 accumulators and kept-token indices bit-exact; fp16 /
+bf16 outputs within max(1 ulp, 2e-3 relative) of the oracle's.
+"""
+import numpy as np
+import pytest
+
+import oracle
+from paper_2509_09090_b200 import workloads as wl
+
+pytestmark = pytest.mark.gpu
+
+torch = pytest.importorskip("torch")
+if torch.cuda.is_available():
+    from paper_2509_09090_b200 import binding as B
+    import gpu_harness as G
+
+
+def bits(a):
+    return np.ascontiguousarray(a, dtype=np.float16).view(np.uint16)
+
+
+KERNELS = [("simt", 1), ("auto", 0)]
+
+
+def _linear_flags():
+    return [0, B.SQAP_L_FORCE_SIMT]
+
+
+def check_linear(x_f16, w_codes, w_scales, rotate=False, row_index=None, up=None, flags_list=None, bf16=False):
+    """Quantize + linear on the GPU vs the oracle; returns the oracle's fp16 output bits."""
+    packed_o, s_o, codes_o = oracle.quantize_act(bits(x_f16), rotate=rotate, row_index=row_index)
+    packed_g, s_g = G.quantize(x_f16, rotate=rotate, row_index=row_index)
+    assert np.array_equal(packed_g, packed_o)
+    assert np.array_equal(s_g, s_o)
+    acc_o = oracle.gemm_i32(codes_o, w_codes)
+    w = G.pack(w_codes, w_scales)
+    if up is None:
+        ref = oracle.epilogue(acc_o, s_o, bits(w_scales), bf16=bf16)
+        wu = None
+    else:
+        acc_u = oracle.gemm_i32(codes_o, up[0])
+        ref = oracle.epilogue_swiglu(acc_o, acc_u, s_o, bits(w_scales), bits(up[1]), bf16=bf16)
+        wu = G.pack(up[0], up[1])
+    for flags in (flags_list if flags_list is not None else _linear_flags()):
+        if up is None:
+            acc_g = G.linear(packed_g, s_g, w, out_dtype=B.SQAP_I32, flags=flags)
+            assert np.array_equal(acc_g, acc_o), f"int32 accumulators differ (flags={flags})"
+        out = G.linear(packed_g, s_g, w, w_up=wu, out_dtype=B.SQAP_BF16 if bf16 else B.SQAP_FP16, flags=flags)
+        ok = G.within_tolerance(out, ref, bf16=bf16)
+        assert ok.all(), f"{(~ok).sum()} outputs outside tolerance (flags={flags})"
+    w.close()
+    if wu:
+        wu.close()
+    return ref
+
+
+# ------------------------------------------------------------------ quantizer
+
+@pytest.mark.parametrize("M,K", [(1, 32), (2, 64), (7, 512), (64, 512), (33, 4096), (5, 11008), (3, 16384),
+                                 (2, 20480), (9, 128), (9, 256)])
+@pytest.mark.parametrize("rotate", [False, True])
+def test_quantizer_bit_exact(M, K, rotate):
+    if rotate and ((K & (K - 1)) or K < 64):
+        pytest.skip("rotation needs a power of two >= 64")
+    x = wl.activations(100 + M, K, M, K, max(1, K // 100), 30.0)
+    x[M // 2] = 0                                              # an all-zero row
+    po, so, _ = oracle.quantize_act(bits(x), rotate=rotate)
+    pg, sg = G.quantize(x, rotate=rotate)
+    assert np.array_equal(pg, po)
+    assert np.array_equal(sg, so)
+
+
+def test_quantizer_row_index_stride_and_empty():
+    x = wl.activations(5, 5, 40, 1024, 10, 30.0)
+    idx = np.array([39, 0, 7, 7, 12], np.int32)
+    po, so, _ = oracle.quantize_act(bits(x), row_index=idx)
+    pg, sg = G.quantize(x, row_index=idx)
+    assert np.array_equal(pg, po) and np.array_equal(sg, so)
+    # a column slice of a wider matrix (the V third of a fused QKV output): ldx = 1024, K = 256 at offset 512
+    sub = np.ascontiguousarray(x[:, 512:768])
+    po, so, _ = oracle.quantize_act(bits(sub), rotate=True)
+    pg, sg = G.quantize(x, rotate=True, K=256, col_offset=512)
+    assert np.array_equal(pg, po) and np.array_equal(sg, so)
+    # M = 0 is a no-op
+    B.sqap_quantize_act(None, 0, 64, 64, None, 0, None, None)
+
+
+def test_quantizer_rejects_bad_arguments():
+    t = torch.zeros(64 * 64, dtype=torch.float16, device="cuda")
+    q = torch.zeros(64 * 32, dtype=torch.uint8, device="cuda")
+    s = torch.zeros(64, dtype=torch.float32, device="cuda")
+    L = B.lib()
+    st = lambda *a: L.sqap_quantize_act(*a, None)
+    assert st(t.data_ptr(), -1, 64, 64, None, 0, q.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
+    assert st(t.data_ptr(), 4, 48, 48, None, 0, q.data_ptr(), s.data_ptr()) == B.SQAP_ERR_ALIGN
+    assert st(t.data_ptr() + 2, 4, 64, 64, None, 0, q.data_ptr(), s.data_ptr()) == B.SQAP_ERR_ALIGN
+    assert st(t.data_ptr(), 4, 96, 96, None, B.SQAP_Q_ROTATE, q.data_ptr(), s.data_ptr()) == B.SQAP_ERR_UNSUPPORTED
+    assert st(t.data_ptr(), 4, 64, 32, None, 0, q.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
+    assert st(None, 4, 64, 64, None, 0, q.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
+
+
+# ------------------------------------------------------------------ weights
+
+@pytest.mark.parametrize("N,K", [(8, 32), (128, 512), (40, 96), (512, 4096), (16, 11008)])
+@pytest.mark.parametrize("on_device", [False, True])
+def test_pack_unpack_round_trip(N, K, on_device):
+    codes = wl.weight_codes(9, N + K, N, K)
+    scales = wl.weight_scales(9, N + K, N)
+    w = G.pack(codes, scales, on_device=on_device)
+    c2, s2 = B.sqap_unpack_weights(w)
+    assert np.array_equal(c2, codes) and np.array_equal(s2.view(np.uint16), scales.view(np.uint16))
+    assert B.sqap_weights_info(w) == (N, K, 0)
+    w.close()
+
+
+def test_pack_rejects_bad_codes_and_scales():
+    codes = wl.weight_codes(9, 1, 16, 64)
+    scales = wl.weight_scales(9, 1, 16)
+    bad = codes.copy()
+    bad[3, 7] = 8
+    with pytest.raises(B.SqapError) as e:
+        G.pack(bad, scales)
+    assert e.value.status == B.SQAP_ERR_RANGE
+    sc = scales.copy()
+    sc[2] = np.float16(0)
+    with pytest.raises(B.SqapError) as e:
+        G.pack(codes, sc)
+    assert e.value.status == B.SQAP_ERR_RANGE
+    sc[2] = np.float16(np.inf)
+    with pytest.raises(B.SqapError) as e:
+        G.pack(codes, sc)
+    assert e.value.status == B.SQAP_ERR_RANGE
+    with pytest.raises(B.SqapError) as e:
+        B.sqap_pack_weights(codes, scales, 16, 48)
+    assert e.value.status == B.SQAP_ERR_ALIGN
+
+
+# ------------------------------------------------------------------ linear: small and ragged shapes
+
+@pytest.mark.parametrize("M,N,K", [(1, 8, 32), (2, 128, 64), (7, 8, 512), (64, 512, 512), (65, 130, 96),
+                                   (9, 72, 11008), (130, 264, 1024), (300, 520, 256)])
+def test_linear_small_shapes(M, N, K):
+    x = wl.activations(20, M * 7 + K, M, K, max(1, K // 100), 20.0)
+    wc = wl.weight_codes(20, N * 3 + K, N, K)
+    ws = wl.weight_scales(20, N * 3 + K, N)
+    check_linear(x, wc, ws)
+    if M <= 8:
+        check_linear(x, wc, ws, flags_list=[B.SQAP_L_FORCE_GEMV])
+
+
+@pytest.mark.parametrize("M", [1, 2, 3, 5, 8])
+def test_gemv_rows_and_swiglu(M):
+    K, N = 4096, 264
+    x = wl.activations(21, M, M, K, 41, 30.0)
+    g = (wl.weight_codes(21, 1, N, K), wl.weight_scales(21, 1, N, mult=0.25))
+    u = (wl.weight_codes(21, 2, N, K), wl.weight_scales(21, 2, N, mult=0.25))
+    check_linear(x, g[0], g[1], flags_list=[B.SQAP_L_FORCE_GEMV, B.SQAP_L_FORCE_SIMT, 0])
+    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_GEMV, B.SQAP_L_FORCE_SIMT, 0])
+
+
+def test_linear_special_operands():
+    K = N = 256
+    x = wl.activations(22, 1, 16, K, 3, 20.0)
+    _, s, codes = oracle.quantize_act(bits(x))
+    pg, sg = G.quantize(x)
+    one = np.float16(1.0)
+    eye = G.pack(np.eye(K, dtype=np.int8), np.full(N, one))
+    for f in _linear_flags():
+        assert np.array_equal(G.linear(pg, sg, eye, out_dtype=B.SQAP_I32, flags=f), codes.astype(np.int32))
+    m8 = G.pack(np.full((N, K), -8, np.int8), np.full(N, one))
+    allm8 = oracle.pack_nibbles(np.full((4, K), -8, np.int8))
+    for f in _linear_flags():
+        assert (G.linear(allm8, np.ones(4, np.float32), m8, out_dtype=B.SQAP_I32, flags=f) == 64 * K).all()
+    p7 = G.pack(np.full((N, K), 7, np.int8), np.full(N, one))
+    for f in _linear_flags():
+        assert (G.linear(allm8, np.ones(4, np.float32), p7, out_dtype=B.SQAP_I32, flags=f) == -56 * K).all()
+
+
+def test_linear_bf16_output_and_padded_rows():
+    M, N, K = 37, 200, 512
+    x = wl.activations(23, 1, M, K, 5, 20.0)
+    wc, ws = wl.weight_codes(23, 2, N, K), wl.weight_scales(23, 2, N)
+    ref = check_linear(x, wc, ws, bf16=True)
+    assert ref.shape == (M, N)
+    pg, sg = G.quantize(x)
+    w = G.pack(wc, ws)
+    a = G.linear(pg, sg, w, ldo=N)
+    b = G.linear(pg, sg, w, ldo=N + 56)
+    assert np.array_equal(a, b)
+    w.close()
+
+
+def test_linear_rejects_bad_arguments():
+    wc, ws = wl.weight_codes(24, 2, 64, 128), wl.weight_scales(24, 2, 64)
+    w = G.pack(wc, ws)
+    w2 = G.pack(wl.weight_codes(24, 3, 32, 128), wl.weight_scales(24, 3, 32))
+    q = torch.zeros(16 * 64, dtype=torch.uint8, device="cuda")
+    s = torch.ones(16, dtype=torch.float32, device="cuda")
+    out = torch.zeros(16 * 64, dtype=torch.float16, device="cuda")
+    ws_t = torch.zeros(1 << 16, dtype=torch.uint8, device="cuda")
+    L = B.lib()
+
+    def call(M=16, w_=w, up=None, o=out.data_ptr(), ldo=64, dt=B.SQAP_FP16, fl=0, wsp=ws_t.data_ptr(), wsb=1 << 16):
+        return L.sqap_w4a4_linear(q.data_ptr(), s.data_ptr(), M, w_.handle, up.handle if up else None, o, ldo, dt, fl,
+                                  wsp, wsb, None)
+
+    assert call() == B.SQAP_OK
+    assert call(M=-1) == B.SQAP_ERR_INVALID
+    assert call(ldo=32) == B.SQAP_ERR_INVALID
+    assert call(up=w2) == B.SQAP_ERR_INVALID
+    assert call(dt=7) == B.SQAP_ERR_INVALID
+    assert call(up=w, dt=B.SQAP_I32) == B.SQAP_ERR_INVALID
+    assert call(o=out.data_ptr() + 2) == B.SQAP_ERR_ALIGN
+    assert call(ldo=68) == B.SQAP_ERR_ALIGN
+    assert call(wsb=128) == B.SQAP_ERR_NOMEM
+    assert call(fl=B.SQAP_L_FORCE_GEMV) == B.SQAP_ERR_UNSUPPORTED
+    assert call(fl=3) == B.SQAP_ERR_INVALID
+    assert call(M=0) == B.SQAP_OK
+    torch.cuda.synchronize()
+    w.close()
+    w2.close()
+
+
+# ------------------------------------------------------------------ pruning
+
+def check_prune(params, scores, centers=None, x=None, out_rows=0):
+    sc = bits(scores) if params["score_rows"] > 0 else scores
+    kept_o, nk_o = oracle.prune_tokens(params, sc, centers)
+    kept_g, nk_g, xo = G.prune(params, scores, centers, x, out_rows)
+    assert np.array_equal(nk_g, nk_o)
+    assert np.array_equal(kept_g, kept_o)
+    if x is not None:
+        xb = bits(x).reshape(params["batch"], params["rows"], -1)
+        ref = oracle.gather_rows(xb, kept_o, nk_o, out_rows)
+        for b in range(params["batch"]):
+            n = min(nk_o[b], out_rows)
+            assert np.array_equal(xo[b, :n], ref[b, :n])
+            assert (xo[b, n:] == 0x7B7B).all()         # rows past n_kept are never written
+    return kept_o, nk_o
+
+
+@pytest.mark.parametrize("k_attn,keep,radius", [(24, 24, -1), (0, 0, -1), (48, 48, -1), (10, 30, 1), (0, 20, 0),
+                                                (5, 48, 2), (60, 10, 1), (0, 100, -1)])
+def test_prune_small_grid(k_attn, keep, radius):
+    c0 = wl.config0()
+    p = wl.prune_params(1, 64, 0, 48, 8, 6, 0, k_attn, keep, ring_radius=radius)
+    check_prune(p, c0["scores"], np.array([[6, 1]], np.int32), c0["x"], 64)
+
+
+def test_prune_batched_full_criterion_and_offgrid_centres():
+    Bn = 16
+    scores = wl.scores_softmax_rows(30, 1, Bn, 32, 256)
+    centers = wl.ring_centers(30, 2, Bn, 16, 16)
+    centers[3] = (-1, 7)
+    centers[4] = (40, 40)
+    centers[5] = (15, 15)
+    x = wl.activations(30, 3, Bn * 288, 512, 5, 30.0)
+    for keep, k_attn, radius in [(64, 32, 1), (128, 64, 1), (192, 96, 2), (154, 40, 1), (128, 128, -1)]:
+        p = wl.prune_params(Bn, 288, 1, 256, 16, 16, 32, k_attn, keep, ring_radius=radius)
+        kept, nk = check_prune(p, scores, centers, x, 32 + keep)
+        assert (nk == 32 + keep).all()
+
+
+def test_prune_ties_large_grid_and_ragged_rows():
+    # many tied scores, a 32x32 grid (the largest supported), rows not a multiple of the block size
+    rng = np.random.default_rng(31)
+    s = rng.integers(0, 6, (2, 1024)).astype(np.float32)
+    p = wl.prune_params(2, 1024 + 77, 50, 1024, 32, 32, 0, 100, 400, ring_radius=3)
+    check_prune(p, s, np.array([[0, 0], [31, 16]], np.int32))
+    s = rng.integers(0, 3, (3, 30)).astype(np.float32)
+    p = wl.prune_params(3, 41, 11, 30, 5, 6, 0, 7, 19, ring_radius=0)
+    check_prune(p, s, np.array([[2, 2], [4, 5], [9, 9]], np.int32))
+    # no visual tokens at all
+    p = wl.prune_params(2, 10, 0, 0, 0, 0, 0, 0, 0)
+    kept, nk, _ = G.prune(p, np.zeros((2, 1), np.float32))
+    assert (nk == 10).all() and (kept == np.arange(10)).all()
+
+
+def test_prune_fps_worked_example():
+    p = wl.prune_params(1, 256, 0, 256, 16, 16, 0, 0, 5)
+    kept, nk, _ = G.prune(p, np.zeros((1, 256), np.float32))
+    assert kept[0, :5].tolist() == [0, 15, 119, 240, 255]
+
+
+def test_prune_rejects_bad_arguments():
+    L = B.lib()
+    k = torch.zeros(64, dtype=torch.int32, device="cuda")
+    n = torch.zeros(1, dtype=torch.int32, device="cuda")
+    s = torch.zeros(48, dtype=torch.float32, device="cuda")
+
+    def call(**kw):
+        d = wl.prune_params(1, 64, 0, 48, 8, 6, 0, 24, 24)
+        d.update(kw)
+        p = B.PruneParams(**d)
+        import ctypes
+        return L.sqap_prune_tokens(ctypes.byref(p), s.data_ptr(), None, None, 0, 0, None, 0, 0, k.data_ptr(),
+                                   n.data_ptr(), None)
+
+    assert call() == B.SQAP_OK
+    assert call(grid_w=7) == B.SQAP_ERR_INVALID
+    assert call(visual_start=20) == B.SQAP_ERR_INVALID
+    assert call(k_attn=-1) == B.SQAP_ERR_INVALID
+    assert call(n_visual=2048, rows=4096, grid_w=64, grid_h=32) == B.SQAP_ERR_UNSUPPORTED
+    torch.cuda.synchronize()
+
+
+# ------------------------------------------------------------------ the five configurations
+
+def test_config0_prune_then_linear():
+    c0 = wl.config0()
+    kept, nk = check_prune(c0["prune"], c0["scores"], None, c0["x"], 40)
+    assert nk[0] == 40
+    idx = kept[0, :40]
+    for rotate in (False, True):
+        check_linear(c0["x"], c0["w_codes"], c0["w_scales"], rotate=rotate, row_index=idx)
+        check_linear(c0["x"], c0["w_codes"], c0["w_scales"], rotate=rotate)
+
+
+def test_config1_attention_projections():
+    c1 = wl.config1()
+    check_linear(c1["x"], c1["wqkv_codes"], c1["wqkv_scales"], rotate=True, flags_list=[0])
+    check_linear(c1["x"], c1["wqkv_codes"], c1["wqkv_scales"], rotate=False, flags_list=[0])
+    check_linear(c1["x_o"], c1["wo_codes"], c1["wo_scales"], flags_list=[0, B.SQAP_L_FORCE_SIMT])
+
+
+def test_config2_pruned_mlp():
+    c2 = wl.config2()
+    kept, nk = check_prune(c2["prune"], c2["scores"], None, c2["x"], 160)
+    assert nk[0] == 160
+    xg = oracle.gather_rows(bits(c2["x"])[None], kept, nk, 160)[0].view(np.float16)
+    # gate/up with the SiLU-gated product fused; the oracle's H then feeds the down projection on both sides
+    h_bits = check_linear(xg, c2["wg_codes"], c2["wg_scales"], up=(c2["wu_codes"], c2["wu_scales"]), flags_list=[0])
+    h = h_bits.view(np.float16)
+    assert np.isfinite(h.astype(np.float32)).all()
+    check_linear(h, c2["wd_codes"], c2["wd_scales"], flags_list=[0])
+
+
+@pytest.mark.parametrize("layer,M", [(0, 288), (31, 160)])
+def test_config3_one_layer_of_the_stack(layer, M):
+    inp = wl.config3_inputs()
+    lw = wl.config3_layer(layer)
+    x = inp["x"]
+    if M == 160:
+        kept, nk = check_prune(inp["prune"], inp["scores"], None, x, 160)
+        x = oracle.gather_rows(bits(x)[None], kept, nk, 160)[0].view(np.float16)
+    qkv = check_linear(x, lw["qkv_codes"], lw["qkv_scales"], rotate=True, flags_list=[0]).view(np.float16)
+    v = np.ascontiguousarray(qkv[:, 8192:])
+    o = check_linear(v, lw["o_codes"], lw["o_scales"], flags_list=[0]).view(np.float16)
+    h = check_linear(o, lw["gate_codes"], lw["gate_scales"], up=(lw["up_codes"], lw["up_scales"]),
+                     flags_list=[0]).view(np.float16)
+    d = check_linear(h, lw["down_codes"], lw["down_scales"], flags_list=[0]).view(np.float16)
+    assert np.isfinite(d.astype(np.float32)).all() and np.abs(d.astype(np.float32)).max() > 0
+
+
+def test_config3_decode_step_gemv():
+    inp = wl.config3_inputs()
+    lw = wl.config3_layer(1)
+    x = inp["x_decode"][:1]
+    qkv = check_linear(x, lw["qkv_codes"], lw["qkv_scales"], rotate=True, flags_list=[0]).view(np.float16)
+    o = check_linear(np.ascontiguousarray(qkv[:, 8192:]), lw["o_codes"], lw["o_scales"], flags_list=[0]).view(np.float16)
+    h = check_linear(o, lw["gate_codes"], lw["gate_scales"], up=(lw["up_codes"], lw["up_scales"]),
+                     flags_list=[0]).view(np.float16)
+    check_linear(h, lw["down_codes"], lw["down_scales"], flags_list=[0])
+
+
+@pytest.mark.parametrize("keep", [64, 192, 256])
+def test_config4_batched_sampled(keep):
+    """Full-size GEMMs (M up to 4608): accumulators checked on sampled entries and on whole sampled rows."""
+    Bn = 16
+    inp = wl.config4_inputs()
+    wts = wl.config4_weights()
+    x = inp["x"].reshape(Bn * 288, 4096)
+    if keep < 256:
+        p = wl.prune_params(Bn, 288, 1, 256, 16, 16, 32, keep // 2, keep, ring_radius=1)
+        kept, nk = check_prune(p, inp["scores"], inp["centers"], x, 32 + keep)
+        xg = oracle.gather_rows(bits(inp["x"]), kept, nk, 32 + keep).reshape(Bn * (32 + keep), 4096).view(np.float16)
+    else:
+        xg = x
+    M = xg.shape[0]
+    po, so, codes = oracle.quantize_act(bits(xg), rotate=True)
+    pg, sg = G.quantize(xg, rotate=True)
+    assert np.array_equal(pg, po) and np.array_equal(sg, so)
+    rng = np.random.default_rng(keep)
+    for name in ("qkv", "gate", "o"):
+        wc, ws = wts[name + "_codes"], wts[name + "_scales"]
+        N = wc.shape[0]
+        w = G.pack(wc, ws)
+        acc = G.linear(pg, sg, w, out_dtype=B.SQAP_I32)
+        out = G.linear(pg, sg, w)
+        rows = np.unique(np.concatenate([[0, M - 1, 255, 256], rng.integers(0, M, 4)]))
+        ref_rows = oracle.gemm_i32(codes[rows], wc)
+        assert np.array_equal(acc[rows], ref_rows)
+        assert G.within_tolerance(out[rows], oracle.epilogue(ref_rows, so[rows], bits(ws))).all()
+        cols = np.unique(np.concatenate([[0, N - 1, 127, 128], rng.integers(0, N, 4)]))
+        ref_cols = oracle.gemm_i32(codes, wc[cols])
+        assert np.array_equal(acc[:, cols], ref_cols)
+        for _ in range(512):
+            m, n = int(rng.integers(0, M)), int(rng.integers(0, N))
+            assert acc[m, n] == oracle.dot_i32(codes[m], wc[n])
+        if name == "gate":
+            wu = G.pack(wts["up_codes"], wts["up_scales"])
+            hs = G.linear(pg, sg, w, w_up=wu)
+            ref_u = oracle.gemm_i32(codes[rows], wts["up_codes"])
+            ref_h = oracle.epilogue_swiglu(ref_rows, ref_u, so[rows], bits(ws), bits(wts["up_scales"]))
+            assert G.within_tolerance(hs[rows], ref_h).all()
+            wu.close()
+        w.close()
