@@ -49,7 +49,7 @@ def linear(packed: np.ndarray, scales: np.ndarray, w: B.Weights, w_up=None, out_
     """Returns the [M, N] output as numpy: uint16 bit patterns for fp16/bf16, int32 for SQAP_I32."""
     M = packed.shape[0]
     N = w.N
-    ldo = ldo or N
+    ldo = ldo or (N + 7) // 8 * 8          # row pitch must be a multiple of 16 bytes
     qd, sd = to_dev(packed), to_dev(scales)
     tdt = torch.int32 if out_dtype == B.SQAP_I32 else torch.int16
     fill = 0x7B7B7B7B if out_dtype == B.SQAP_I32 else 0x7B7B
