@@ -150,6 +150,18 @@ def test_linear_small_shapes(M, N, K):
         check_linear(x, wc, ws, flags_list=[B.SQAP_L_FORCE_GEMV])
 
 
+@pytest.mark.parametrize("M,N,K,swiglu", [(16, 128, 128, False), (9, 8, 256, False), (257, 130, 384, False),
+                                          (144, 320, 1024, False), (700, 200, 512, False), (40, 192, 512, True),
+                                          (300, 64, 256, True), (513, 448, 1152, True), (17, 1088, 11008, False)])
+def test_linear_tcgen05_forced(M, N, K, swiglu):
+    """The tensor-core kernel on shapes with ragged token tiles, partial weight tiles and the fused gate."""
+    x = wl.activations(25, M + K, M, K, max(1, K // 100), 20.0)
+    g = (wl.weight_codes(25, N + K, N, K), wl.weight_scales(25, N + K, N, mult=0.5))
+    u = (wl.weight_codes(25, N + K + 1, N, K), wl.weight_scales(25, N + K + 1, N, mult=0.5)) if swiglu else None
+    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05])
+    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05], bf16=True)
+
+
 @pytest.mark.parametrize("M", [1, 2, 3, 5, 8])
 def test_gemv_rows_and_swiglu(M):
     K, N = 4096, 264
