@@ -396,6 +396,49 @@ def run_reference(args):
     }))
 
 
+def run_single_kernel(args):
+    """Profiling aid: a few launches of one kernel of the path on a small, larger-than-L2 case
+    (what `ncu -k ... -c 3` captures). Prints nothing that counts as a bench value."""
+    import torch
+    from paper_2509_09090_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    M, H = M_FULL, wl.HIDDEN
+    x = torch.from_numpy(wl.config4_inputs(seed=4, batch=N_OBS)["x"].reshape(M, H)).to(dev)
+    q = torch.empty(M * wl.FFN // 2, dtype=torch.uint8, device=dev)
+    sx = torch.empty(M, dtype=torch.float32, device=dev)
+    if args.kernel == "quantize":
+        for i in range(args.steps):
+            B.sqap_quantize_act(x, M, H, H, None, B.SQAP_Q_ROTATE if i % 2 == 0 else 0, q, sx)
+    elif args.kernel in ("gemm", "gemv", "swiglu"):
+        names = {"gemm": ("qkv",), "gemv": ("qkv",), "swiglu": ("gate", "up")}[args.kernel]
+        wts = wl.config4_weights(seed=4)
+        ws = [B.sqap_pack_weights(np.ascontiguousarray(wts[n + "_codes"]), np.ascontiguousarray(wts[n + "_scales"]),
+                                  wts[n + "_codes"].shape[0], H) for n in names]
+        Mk = 1 if args.kernel == "gemv" else M
+        N = ws[0].N
+        out = torch.empty(Mk, N, dtype=torch.float16, device=dev)
+        nb = B.sqap_workspace_bytes(Mk, N, H)
+        wsp = torch.empty(nb, dtype=torch.uint8, device=dev)
+        B.sqap_quantize_act(x, Mk, H, H, None, B.SQAP_Q_ROTATE, q, sx)
+        for i in range(args.steps):
+            B.sqap_w4a4_linear(q, sx, Mk, ws[0], ws[1] if len(ws) > 1 else None, out, N, B.SQAP_FP16,
+                               B.SQAP_L_REUSE_EXPANDED if i else 0, wsp, nb)
+    elif args.kernel == "prune":
+        inp = wl.config4_inputs(seed=4, batch=N_OBS)
+        sc, ce = torch.from_numpy(inp["scores"]).to(dev), torch.from_numpy(inp["centers"]).to(dev)
+        x1 = torch.empty(M_PRUNED, H, dtype=torch.float16, device=dev)
+        kept = torch.empty(N_OBS, wl.ROWS, dtype=torch.int32, device=dev)
+        nk = torch.empty(N_OBS, dtype=torch.int32, device=dev)
+        p = wl.prune_params(N_OBS, wl.ROWS, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32, K_ATTN, KEEP,
+                            ring_radius=RING_RADIUS)
+        for i in range(args.steps):
+            B.sqap_prune_tokens(p, sc, ce, x, H, H, x1, H, ROWS_KEPT, kept, nk)
+    torch.cuda.synchronize()
+    assert B.sqap_device_status() == B.SQAP_OK
+    print(json.dumps({"profiling_run": args.kernel, "launches": B.sqap_kernel_launch_count()}))
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -403,8 +446,12 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "quantize", "prune"],
+                    help="profiling aid: launch only this kernel --steps times (no bench line)")
     args = ap.parse_args()
-    if args.impl == "reference":
+    if args.kernel:
+        run_single_kernel(args)
+    elif args.impl == "reference":
         run_reference(args)
     else:
         run_ours(args)
