@@ -121,6 +121,48 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return static_cast<uint64_t>((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
 
+// One finished accumulator tile -> global memory. The thread owns output channel n (one TMEM lane) and
+// walks the tile's tokens 16 at a time; the per-token bias sums and scales of a chunk are fetched by
+// lanes 0-15 with one coalesced load each (one chunk ahead) and broadcast by shuffle.
+template <int OUT, bool SWIGLU>
+__device__ __forceinline__ void epilogue_tile(const Args& a, uint32_t taddr, int m0, int n, bool n_ok, float sw, int lane) {
+    constexpr int ESZ = OUT == SQAP_I32 ? 4 : 2;
+    const int ml = lane & 15;
+    const int64_t row_bytes = a.ldo * ESZ;
+    int mm = m0 + ml;
+    int bs_next = mm < a.M ? (__ldg(a.bias_sum + mm) << 7) : 0;
+    float sx_next = mm < a.M ? __ldg(a.act_scales + mm) : 0.0f;
+    const bool writer = n_ok && (!SWIGLU || (lane & 1) == 0);
+    for (int c = 0; c < a.BN; c += 16) {
+        uint32_t v[16];
+        tc_ld16(taddr + c, v);
+        const int bs_cur = bs_next;
+        const float sx_cur = sx_next;
+        mm = m0 + c + 16 + ml;
+        if (c + 16 < a.BN) {
+            bs_next = mm < a.M ? (__ldg(a.bias_sum + mm) << 7) : 0;
+            sx_next = mm < a.M ? __ldg(a.act_scales + mm) : 0.0f;
+        }
+        tc_wait_ld();
+        const int valid = a.M - (m0 + c);  // tokens of this chunk that exist
+        uint8_t* optr = static_cast<uint8_t*>(a.out) + static_cast<int64_t>(m0 + c) * row_bytes + static_cast<int64_t>(n) * ESZ;
+#pragma unroll
+        for (int j = 0; j < 16; ++j) {
+            const int bs = __shfl_sync(0xffffffffu, bs_cur, j);
+            const float sx = __shfl_sync(0xffffffffu, sx_cur, j);
+            const int t = (static_cast<int>(v[j]) - bs) >> 4;
+            float y = __fmul_rn(__fmul_rn(static_cast<float>(t), sx), sw);
+            if (SWIGLU) y = swiglu(y, __shfl_xor_sync(0xffffffffu, y, 1));  // even lane: gate, odd lane: up
+            if (writer && j < valid) {
+                if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(optr) = __float2half_rn(y);
+                else if (OUT == SQAP_BF16) *reinterpret_cast<__nv_bfloat16*>(optr) = __float2bfloat16_rn(y);
+                else *reinterpret_cast<int32_t*>(optr) = t;
+            }
+            optr += row_bytes;
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------- the kernel
 __global__ void __launch_bounds__(THREADS, 1)
 w4a4_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_w_up,
@@ -233,6 +275,9 @@ w4a4_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             for (int ks = 0; ks < k_steps; ++ks, ++it) {
                 const int s = it % STAGES;
                 if (!__all_sync(0xffffffffu, mbar_wait(full(s), (it / STAGES) & 1u, abort_flag))) { failed = true; break; }
+#ifdef SQAP_EXP_NO_UNPACK
+                fence_proxy_async(); mbar_arrive(ufull(s)); continue;
+#endif
                 const uint8_t* src = sm + OFF_WP + s * WP_BYTES + r * 64;
                 uint8_t* dst = sm + OFF_WU + s * WU_BYTES + dr * 128;
 #pragma unroll
@@ -272,24 +317,16 @@ w4a4_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
                 n_ok = n < a.N;
                 sw = n_ok ? __half2float(a.w_scales[n]) : 0.0f;
             }
-            for (int c = 0; c < a.BN; c += 16) {
-                uint32_t v[16];
-                tc_ld16(taddr + c, v);
-                tc_wait_ld();
-#pragma unroll
-                for (int j = 0; j < 16; ++j) {
-                    const int m = m0 + c + j;
-                    if (m >= a.M) break;  // uniform across the warp
-                    const int t = finish_acc(static_cast<int>(v[j]), __ldg(a.bias_sum + m));
-                    float y = dequant(t, __ldg(a.act_scales + m), sw);
-                    if (a.swiglu) {
-                        const float other = __shfl_xor_sync(0xffffffffu, y, 1);
-                        y = swiglu(y, other);  // meaningful on even lanes: y = gate, other = up
-                        if ((row & 1) == 0 && n_ok) store_out(a.out, static_cast<int64_t>(m) * a.ldo + n, a.out_dtype, y, t);
-                    } else if (n_ok) {
-                        store_out(a.out, static_cast<int64_t>(m) * a.ldo + n, a.out_dtype, y, t);
-                    }
-                }
+#ifdef SQAP_EXP_NO_EPI
+            tc_fence_before(); mbar_arrive(acc_empty(b)); continue;
+#endif
+            if (a.swiglu) {
+                if (a.out_dtype == SQAP_FP16) epilogue_tile<SQAP_FP16, true>(a, taddr, m0, n, n_ok, sw, lane);
+                else epilogue_tile<SQAP_BF16, true>(a, taddr, m0, n, n_ok, sw, lane);
+            } else {
+                if (a.out_dtype == SQAP_FP16) epilogue_tile<SQAP_FP16, false>(a, taddr, m0, n, n_ok, sw, lane);
+                else if (a.out_dtype == SQAP_BF16) epilogue_tile<SQAP_BF16, false>(a, taddr, m0, n, n_ok, sw, lane);
+                else epilogue_tile<SQAP_I32, false>(a, taddr, m0, n, n_ok, sw, lane);
             }
             tc_fence_before();
             mbar_arrive(acc_empty(b));
