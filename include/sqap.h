@@ -36,7 +36,8 @@ typedef enum {
     SQAP_ERR_UNSUPPORTED = 4, /* e.g. rotation with K not a power of two; n_visual > 1024 */
     SQAP_ERR_NOMEM = 5,       /* device allocation failed, or workspace too small */
     SQAP_ERR_CUDA = 6,        /* a CUDA call failed; see sqap_last_cuda_error() */
-    SQAP_ERR_TIMEOUT = 7      /* a bounded wait inside a kernel ran out (reported by sqap_device_status) */
+    SQAP_ERR_TIMEOUT = 7,     /* a bounded wait inside a kernel ran out (reported by sqap_device_status) */
+    SQAP_ERR_TOO_LARGE = 8    /* the problem does not fit a fixed-size resource (sqap_w4a4_linear_static) */
 } sqap_status;
 
 /* Output element types of sqap_w4a4_linear. */
@@ -118,6 +119,35 @@ size_t sqap_workspace_bytes(int M, int N, int K, uint32_t flags);
 sqap_status sqap_w4a4_linear(const uint8_t* q_packed, const float* act_scales, int M, const sqap_weights* w,
                              const sqap_weights* w_up, void* out, int64_t ldo, int out_dtype, uint32_t flags,
                              void* workspace, size_t workspace_bytes, void* stream);
+
+/*
+ * The same linear for callers that must not allocate. (The paper has no counterpart: this entry point
+ * exists only for the sake of such callers.)
+ *
+ * Who needs it: code that runs where device allocation is forbidden or would be harmful — a real-time
+ * control loop that may not touch the allocator between robot actions, a process whose device memory
+ * has all been handed to another component's pool, a host runtime that gives the library a fixed memory
+ * budget and nothing more. Those callers
+ * cannot size and cudaMalloc the workspace that sqap_w4a4_linear asks for, so here the scratch is an
+ * array of SQAP_STATIC_WORKSPACE_BYTES bytes built into the library image (every GPU that loads the
+ * library holds that much until the process exits). Inputs and outputs are still the caller's.
+ *
+ * Semantics, results and argument rules are exactly those of sqap_w4a4_linear; the differences:
+ *   - no workspace arguments, and SQAP_L_REUSE_EXPANDED is rejected (INVALID);
+ *   - the problem must satisfy sqap_workspace_bytes(M, N, K, flags) <= SQAP_STATIC_WORKSPACE_BYTES
+ *     (about M * K <= 4 Mi, e.g. 288 rows at K = 11008 or 1020 rows at K = 4096); anything larger
+ *     returns SQAP_ERR_TOO_LARGE and launches nothing;
+ *   - the call itself calls no cudaMalloc / cudaFree and no allocating library routine;
+ *   - the FIRST call on each device looks up the array's device address (a one-time query, with that
+ *     device current); make that first call during set-up, before any stream capture begins;
+ *   - all calls on a device share the one array, which simply keeps what the last call left in it (no
+ *     part of it has to be cleared: each call rewrites everything it reads). Two calls whose kernels can
+ *     overlap on the GPU — different streams, no dependency between them — race on it; serialise them.
+ */
+#define SQAP_STATIC_WORKSPACE_BYTES (4 * 1024 * 1024 + 8192)
+sqap_status sqap_w4a4_linear_static(const uint8_t* q_packed, const float* act_scales, int M, const sqap_weights* w,
+                                    const sqap_weights* w_up, void* out, int64_t ldo, int out_dtype, uint32_t flags,
+                                    void* stream);
 
 /*
  * Parameters of the pruning criterion (Section "Quantization-aware Pruning Strategies").

@@ -12,14 +12,16 @@ _HERE = os.path.dirname(os.path.abspath(__file__))
 LIB_PATH = os.path.join(_HERE, "libsqap.so")
 
 SQAP_OK, SQAP_ERR_INVALID, SQAP_ERR_RANGE, SQAP_ERR_ALIGN, SQAP_ERR_UNSUPPORTED, SQAP_ERR_NOMEM, \
-    SQAP_ERR_CUDA, SQAP_ERR_TIMEOUT = range(8)
+    SQAP_ERR_CUDA, SQAP_ERR_TIMEOUT, SQAP_ERR_TOO_LARGE = range(9)
+SQAP_STATIC_WORKSPACE_BYTES = 4 * 1024 * 1024 + 8192
 SQAP_FP16, SQAP_BF16, SQAP_I32 = 0, 1, 2
 SQAP_Q_ROTATE = 1
 SQAP_W_ROTATED = 1
 SQAP_L_FORCE_SIMT, SQAP_L_FORCE_TCGEN05, SQAP_L_FORCE_GEMV, SQAP_L_REUSE_EXPANDED = 1, 2, 4, 8
 
 EXPORTS = ("sqap_pack_weights", "sqap_free_weights", "sqap_weights_info", "sqap_unpack_weights",
-           "sqap_quantize_act", "sqap_workspace_bytes", "sqap_w4a4_linear", "sqap_prune_tokens",
+           "sqap_quantize_act", "sqap_workspace_bytes", "sqap_w4a4_linear", "sqap_w4a4_linear_static",
+           "sqap_prune_tokens",
            "sqap_project_center", "sqap_device_status", "sqap_last_cuda_error", "sqap_status_string",
            "sqap_kernel_launch_count")
 
@@ -59,6 +61,7 @@ def lib() -> ctypes.CDLL:
     L.sqap_workspace_bytes.argtypes = [i32, i32, i32, u32]
     L.sqap_workspace_bytes.restype = sz
     L.sqap_w4a4_linear.argtypes = [vp, vp, i32, vp, vp, vp, i64, i32, u32, vp, sz, vp]
+    L.sqap_w4a4_linear_static.argtypes = [vp, vp, i32, vp, vp, vp, i64, i32, u32, vp]
     L.sqap_prune_tokens.argtypes = [ctypes.POINTER(PruneParams), vp, vp, vp, i64, i32, vp, i64, i32, vp, vp, vp]
     L.sqap_project_center.argtypes = [ctypes.POINTER(ctypes.c_double)] * 3 + [ctypes.c_double, ctypes.c_double,
                                                                               ctypes.POINTER(ctypes.c_int32),
@@ -159,6 +162,15 @@ def sqap_w4a4_linear(q_packed, act_scales, M: int, w: Weights, w_up, out, ldo: i
     _check(lib().sqap_w4a4_linear(_ptr(q_packed), _ptr(act_scales), M, w.handle, w_up.handle if w_up else None,
                                   _ptr(out), ldo, out_dtype, flags, _ptr(workspace), workspace_bytes,
                                   _stream(stream)), "sqap_w4a4_linear")
+
+
+def sqap_w4a4_linear_static(q_packed, act_scales, M: int, w: Weights, w_up, out, ldo: int, out_dtype: int, flags: int,
+                            stream=None):
+    """The linear without a caller workspace, for callers that cannot allocate device memory: the scratch
+    is a fixed array inside the library (see include/sqap.h for its size limit and sharing rules)."""
+    _check(lib().sqap_w4a4_linear_static(_ptr(q_packed), _ptr(act_scales), M, w.handle,
+                                         w_up.handle if w_up else None, _ptr(out), ldo, out_dtype, flags,
+                                         _stream(stream)), "sqap_w4a4_linear_static")
 
 
 def sqap_prune_tokens(params: dict, scores, ring_center, x, ldx: int, K: int, x_out, ldo: int, out_rows: int,

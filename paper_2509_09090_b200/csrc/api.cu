@@ -72,6 +72,7 @@ const char* sqap_status_string(sqap_status s) {
         case SQAP_ERR_NOMEM: return "out of memory or workspace too small";
         case SQAP_ERR_CUDA: return "CUDA error";
         case SQAP_ERR_TIMEOUT: return "bounded device wait expired";
+        case SQAP_ERR_TOO_LARGE: return "problem too large for the built-in scratch array";
     }
     return "unknown status";
 }

@@ -33,8 +33,8 @@ def test_library_exports_every_declared_symbol():
 
 def test_status_strings_and_counters():
     L = B.lib()
-    seen = {L.sqap_status_string(i).decode() for i in range(8)}
-    assert len(seen) == 8 and "ok" in seen
+    seen = {L.sqap_status_string(i).decode() for i in range(9)}
+    assert len(seen) == 9 and "ok" in seen
     assert L.sqap_status_string(99).decode() == "unknown status"
     assert L.sqap_kernel_launch_count() >= 0
 
