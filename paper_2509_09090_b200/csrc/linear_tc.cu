@@ -9,7 +9,7 @@
 //   warps 2-5   unpack: packed nibbles -> two int8 vectors by masking alone (see common.cuh), written
 //               in the 128B-swizzled K-major layout the MMA reads; 2 logic ops per 8 weights
 //   warp 1      MMA issuer: 4 x tcgen05.mma (K = 32 each) per K-step into one of two TMEM accumulators
-//   warps 6-9   epilogue: tcgen05.ld the finished accumulator, remove the nibble bias, apply both
+//   warps 6-13  epilogue: tcgen05.ld the finished accumulator, remove the nibble bias, apply both
 //               scales (or SwiGLU), store; overlaps the next tile's main loop
 // Every wait on an mbarrier is bounded; on expiry the kernel records SQAP_ERR_TIMEOUT in the device
 // status word, drains and frees its tensor memory, and returns.
@@ -32,7 +32,8 @@ constexpr int OFF_WU = OFF_X + STAGES * X_BYTES;
 constexpr int OFF_WP = OFF_WU + STAGES * WU_BYTES;
 constexpr int OFF_BAR = OFF_WP + STAGES * WP_BYTES;
 constexpr int SMEM_BYTES = OFF_BAR + 256 + 1024;  // barriers + slack for 1024-byte alignment
-constexpr int THREADS = 320;
+constexpr int EPI_WARPS = 8;                 // two per TMEM lane quadrant, each takes half of the tile's tokens
+constexpr int THREADS = 32 * (6 + EPI_WARPS);
 constexpr long long WAIT_LIMIT_CLOCKS = 4000000000LL;  // ~2 s
 
 struct Args {
@@ -121,44 +122,71 @@ __device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
     return static_cast<uint64_t>((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
 }
 
-// One finished accumulator tile -> global memory. The thread owns output channel n (one TMEM lane) and
-// walks the tile's tokens 16 at a time; the per-token bias sums and scales of a chunk are fetched by
-// lanes 0-15 with one coalesced load each (one chunk ahead) and broadcast by shuffle.
+__device__ __forceinline__ float silu_mul_fast(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
+
+// Part of one finished accumulator tile -> global memory. The thread owns one TMEM lane (output channel n;
+// with SwiGLU the even lane of a pair holds the gate and the odd lane the up projection of channel n) and
+// walks the tokens [c_begin, c_end) of the tile 16 at a time; the per-token bias sums and scales of a chunk
+// are fetched by lanes 0-15 with one coalesced load each (one chunk ahead) and broadcast by shuffle.
 template <int OUT, bool SWIGLU>
-__device__ __forceinline__ void epilogue_tile(const Args& a, uint32_t taddr, int m0, int n, bool n_ok, float sw, int lane) {
+__device__ __forceinline__ void epilogue_tile(const Args& a, uint32_t taddr, int m0, int c_begin, int c_end, int n,
+                                              bool n_ok, float sw, int lane) {
     constexpr int ESZ = OUT == SQAP_I32 ? 4 : 2;
     const int ml = lane & 15;
+    const bool odd = (lane & 1) != 0;
     const int64_t row_bytes = a.ldo * ESZ;
-    int mm = m0 + ml;
+    int mm = m0 + c_begin + ml;
     int bs_next = mm < a.M ? (__ldg(a.bias_sum + mm) << 7) : 0;
     float sx_next = mm < a.M ? __ldg(a.act_scales + mm) : 0.0f;
-    const bool writer = n_ok && (!SWIGLU || (lane & 1) == 0);
-    for (int c = 0; c < a.BN; c += 16) {
+    for (int c = c_begin; c < c_end; c += 16) {
         uint32_t v[16];
         tc_ld16(taddr + c, v);
         const int bs_cur = bs_next;
         const float sx_cur = sx_next;
         mm = m0 + c + 16 + ml;
-        if (c + 16 < a.BN) {
+        if (c + 16 < c_end) {
             bs_next = mm < a.M ? (__ldg(a.bias_sum + mm) << 7) : 0;
             sx_next = mm < a.M ? __ldg(a.act_scales + mm) : 0.0f;
         }
         tc_wait_ld();
         const int valid = a.M - (m0 + c);  // tokens of this chunk that exist
         uint8_t* optr = static_cast<uint8_t*>(a.out) + static_cast<int64_t>(m0 + c) * row_bytes + static_cast<int64_t>(n) * ESZ;
+        if (SWIGLU) {
+            // Columns are handled in pairs: the even lane finishes column j (needs the up value of its
+            // partner), the odd lane column j+1 (needs the gate value of its partner): one exchange per pair.
 #pragma unroll
-        for (int j = 0; j < 16; ++j) {
-            const int bs = __shfl_sync(0xffffffffu, bs_cur, j);
-            const float sx = __shfl_sync(0xffffffffu, sx_cur, j);
-            const int t = (static_cast<int>(v[j]) - bs) >> 4;
-            float y = __fmul_rn(__fmul_rn(static_cast<float>(t), sx), sw);
-            if (SWIGLU) y = swiglu(y, __shfl_xor_sync(0xffffffffu, y, 1));  // even lane: gate, odd lane: up
-            if (writer && j < valid) {
-                if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(optr) = __float2half_rn(y);
-                else if (OUT == SQAP_BF16) *reinterpret_cast<__nv_bfloat16*>(optr) = __float2bfloat16_rn(y);
-                else *reinterpret_cast<int32_t*>(optr) = t;
+            for (int j = 0; j < 16; j += 2) {
+                const float y0 = __fmul_rn(__fmul_rn(static_cast<float>((static_cast<int>(v[j]) - __shfl_sync(0xffffffffu, bs_cur, j)) >> 4),
+                                                     __shfl_sync(0xffffffffu, sx_cur, j)), sw);
+                const float y1 = __fmul_rn(__fmul_rn(static_cast<float>((static_cast<int>(v[j + 1]) - __shfl_sync(0xffffffffu, bs_cur, j + 1)) >> 4),
+                                                     __shfl_sync(0xffffffffu, sx_cur, j + 1)), sw);
+                const float got = __shfl_xor_sync(0xffffffffu, odd ? y0 : y1, 1);
+                const float h = odd ? silu_mul_fast(got, y1) : silu_mul_fast(y0, got);
+                const int jj = odd ? j + 1 : j;
+                if (n_ok && jj < valid) {
+                    uint8_t* o = optr + jj * row_bytes;
+                    if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(h);
+                    else *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(h);
+                }
             }
-            optr += row_bytes;
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int bs = __shfl_sync(0xffffffffu, bs_cur, j);
+                const float sx = __shfl_sync(0xffffffffu, sx_cur, j);
+                const int t = (static_cast<int>(v[j]) - bs) >> 4;
+                const float y = __fmul_rn(__fmul_rn(static_cast<float>(t), sx), sw);
+#ifndef SQAP_EXP_NO_STORE
+                if (n_ok && j < valid) {
+                    if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(optr) = __float2half_rn(y);
+                    else if (OUT == SQAP_BF16) *reinterpret_cast<__nv_bfloat16*>(optr) = __float2bfloat16_rn(y);
+                    else *reinterpret_cast<int32_t*>(optr) = t;
+                }
+#else
+                if (y == 123.456f && n_ok) *reinterpret_cast<int32_t*>(optr) = t;
+#endif
+                optr += row_bytes;
+            }
         }
     }
 }
@@ -193,7 +221,7 @@ w4a4_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full(b), 1);
-            mbar_init(acc_empty(b), 128);
+            mbar_init(acc_empty(b), 32 * EPI_WARPS);
         }
         abort_flag[0] = 0;
         abort_flag[1] = 0;  // always-zero word for waits that must ignore the abort request
@@ -298,6 +326,9 @@ w4a4_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
         // ---------------- epilogue warps: warp % 4 selects the 32-lane quadrant of tensor memory
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
+        const int split = ((a.BN / 16 + 1) / 2) * 16;  // first token of the second half of the tile
+        const int c_begin = (warp - 6) < 4 ? 0 : (EPI_WARPS == 8 ? split : 0);
+        const int c_end = (EPI_WARPS == 8 && (warp - 6) < 4) ? split : a.BN;
         uint32_t lt = 0;
         for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x, ++lt) {
             const int b = lt & 1;
@@ -321,12 +352,12 @@ w4a4_tc_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__
             tc_fence_before(); mbar_arrive(acc_empty(b)); continue;
 #endif
             if (a.swiglu) {
-                if (a.out_dtype == SQAP_FP16) epilogue_tile<SQAP_FP16, true>(a, taddr, m0, n, n_ok, sw, lane);
-                else epilogue_tile<SQAP_BF16, true>(a, taddr, m0, n, n_ok, sw, lane);
+                if (a.out_dtype == SQAP_FP16) epilogue_tile<SQAP_FP16, true>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
+                else epilogue_tile<SQAP_BF16, true>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
             } else {
-                if (a.out_dtype == SQAP_FP16) epilogue_tile<SQAP_FP16, false>(a, taddr, m0, n, n_ok, sw, lane);
-                else if (a.out_dtype == SQAP_BF16) epilogue_tile<SQAP_BF16, false>(a, taddr, m0, n, n_ok, sw, lane);
-                else epilogue_tile<SQAP_I32, false>(a, taddr, m0, n, n_ok, sw, lane);
+                if (a.out_dtype == SQAP_FP16) epilogue_tile<SQAP_FP16, false>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
+                else if (a.out_dtype == SQAP_BF16) epilogue_tile<SQAP_BF16, false>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
+                else epilogue_tile<SQAP_I32, false>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
             }
             tc_fence_before();
             mbar_arrive(acc_empty(b));
