@@ -158,7 +158,7 @@ class Path:
         self.ddec = t.empty(N_OBS, wl.HIDDEN, dtype=f16, device=device)
         self.kept = t.empty(N_OBS, wl.ROWS, dtype=i32, device=device)
         self.nkept = t.empty(N_OBS, dtype=i32, device=device)
-        self.ws_bytes = B.sqap_workspace_bytes(M, wl.QKV, wl.FFN)
+        self.ws_bytes = B.sqap_quantize_linear_workspace_bytes(M, wl.QKV, wl.FFN)
         self.ws = t.empty(self.ws_bytes, dtype=u8, device=device)
         assert self.ws.data_ptr() % 256 == 0
         self.prune_params = wl.prune_params(N_OBS, wl.ROWS, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32,
@@ -173,8 +173,8 @@ class Path:
 
     def linear(self, x_ptr, M, K, ldx, w, w_up, out, rotate=False, flags=0):
         B = self.B
-        B.sqap_quantize_act(x_ptr, M, K, ldx, None, B.SQAP_Q_ROTATE if rotate else 0, self.q, self.sx)
-        B.sqap_w4a4_linear(self.q, self.sx, M, w, w_up, out, out.shape[1], B.SQAP_FP16, flags, self.ws, self.ws_bytes)
+        B.sqap_quantize_linear(x_ptr, M, ldx, None, B.SQAP_Q_ROTATE if rotate else 0, w, w_up, out, out.shape[1],
+                               B.SQAP_FP16, flags, self.ws, self.ws_bytes)
 
     def layer(self, x, M, L: Layer, d_out):
         H = wl.HIDDEN
@@ -396,6 +396,146 @@ def run_reference(args):
     }))
 
 
+def graph_time_us(torch, launch, reps: int, replays: int = 5) -> float:
+    """Average device time of one `launch(i)`: `reps` launches (i = 0 .. reps-1, rotating buffers) captured
+    into one CUDA graph, replayed, timed with events on the replay stream; best of `replays`."""
+    st = torch.cuda.Stream()
+    with torch.cuda.stream(st):
+        for i in range(min(reps, 3)):
+            launch(i)
+        st.synchronize()
+        g = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(g, stream=st):
+            for i in range(reps):
+                launch(i)
+        g.replay()
+        st.synchronize()
+        best = float("inf")
+        for _ in range(replays):
+            a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
+            a.record(st)
+            g.replay()
+            b.record(st)
+            st.synchronize()
+            best = min(best, a.elapsed_time(b))
+    return best * 1e3 / reps
+
+
+def kernel_table(torch, B, peaks, device):
+    """Every kernel of the path timed alone at the workload's shapes, against the roofline that bounds it.
+    Buffers rotate through more than the L2 capacity, so the HBM figures are DRAM figures. Weights for this
+    table are random codes generated on the device (timing does not depend on their values)."""
+    t = torch
+    H, F, Q = wl.HIDDEN, wl.FFN, wl.QKV
+    hbm = peaks["hbm_gbs"]
+    tpk = 2.0 * peaks["bf16"]
+    rows = []
+    L2 = 160e6   # rotate through at least this many bytes
+
+    def ncopies(nbytes):
+        return max(2, int(np.ceil(L2 / max(nbytes, 1))))
+
+    def add(name, shape, bound, work, us, note=""):
+        if bound == "hbm":
+            ach = work / (us * 1e-6) / 1e9
+            rows.append(dict(kernel=name, shape=shape, bound="hbm", bytes=work, us=round(us, 2), achieved_gbs=round(ach, 1),
+                             frac=round(ach / hbm, 3), note=note))
+        elif bound == "tensor":
+            ach = work / (us * 1e-6) / 1e12
+            rows.append(dict(kernel=name, shape=shape, bound="tensor", ops=work, us=round(us, 2), achieved_tops=round(ach, 1),
+                             frac=round(ach / tpk, 3), note=note))
+        else:
+            rows.append(dict(kernel=name, shape=shape, bound=bound, us=round(us, 2), note=note))
+
+    gen = t.Generator(device=device)
+    gen.manual_seed(1234)
+
+    def rand_x(M, K):
+        return (t.randn(M, K, device=device, generator=gen) * 1.0).to(t.float16)
+
+    def rand_w(N, K):
+        codes = t.randint(-8, 8, (N, K), dtype=t.int8, device=device, generator=gen)
+        scales = (t.rand(N, device=device, generator=gen) * 0.015 + 0.005).to(t.float16)
+        w = B.sqap_pack_weights(codes, scales, N, K)
+        t.cuda.synchronize()
+        return w
+
+    # ---- quantizer (public nibble output) and the fused form (expanded output is timed inside the linears)
+    for (M, K, rot) in ((4608, H, True), (4608, H, False), (4608, F, False), (2560, H, True), (288, H, True),
+                        (160, F, False), (16, H, False)):
+        nb = M * K * 2.5 + 4 * M
+        n = ncopies(M * K * 2)
+        xs = [rand_x(M, K) for _ in range(n)]
+        q = t.empty(M * K // 2, dtype=t.uint8, device=device)
+        sx = t.empty(M, dtype=t.float32, device=device)
+        fl = B.SQAP_Q_ROTATE if rot else 0
+        us = graph_time_us(t, lambda i: B.sqap_quantize_act(xs[i % n], M, K, K, None, fl, q, sx), reps=max(n, 8))
+        add("quantize_act" + ("+hadamard" if rot else ""), f"M={M} K={K}", "hbm", nb, us)
+        del xs
+
+    # ---- gather (prune compaction) and the criterion
+    inp = wl.config4_inputs(seed=4, batch=N_OBS)
+    sc, ce = t.from_numpy(inp["scores"]).to(device), t.from_numpy(inp["centers"]).to(device)
+    n = ncopies(M_FULL * H * 2)
+    xs = [rand_x(M_FULL, H) for _ in range(n)]
+    x1 = t.empty(M_PRUNED, H, dtype=t.float16, device=device)
+    kept = t.empty(N_OBS, wl.ROWS, dtype=t.int32, device=device)
+    nk = t.empty(N_OBS, dtype=t.int32, device=device)
+    p = wl.prune_params(N_OBS, wl.ROWS, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32, K_ATTN, KEEP,
+                        ring_radius=RING_RADIUS)
+    us_sel = graph_time_us(t, lambda i: B.sqap_prune_tokens(p, sc, ce, None, 0, 0, None, 0, 0, kept, nk), reps=8)
+    us_all = graph_time_us(t, lambda i: B.sqap_prune_tokens(p, sc, ce, xs[i % n], H, H, x1, H, ROWS_KEPT, kept, nk),
+                           reps=max(n, 8))
+    add("prune_select (top-k U ring U FPS, compaction)", f"16 obs x 256 visual -> {KEEP}", "latency", 0, us_sel,
+        note=f"{KEEP - K_ATTN} or fewer dependent FPS steps per observation")
+    add("gather_rows", f"16 x {ROWS_KEPT} rows x {H}", "hbm", 2 * M_PRUNED * H * 2, max(us_all - us_sel, 1e-3),
+        note="prune call minus the selection kernel")
+    del xs
+
+    # ---- linears: fused quantize + GEMM is what a layer runs; the GEMM alone via REUSE_EXPANDED
+    shapes = (("qkv", Q, H, False), ("o", H, H, False), ("gate_up_swiglu", F, H, True), ("down", H, F, False))
+    for (nm, N, K, sw) in shapes:
+        wbytes = N * K // 2 * (2 if sw else 1)
+        n = ncopies(wbytes)
+        ws = [(rand_w(N, K), rand_w(N, K) if sw else None) for _ in range(n)]
+        for M in (4608, 2560, 288, 160, 16, 1):
+            x = rand_x(M, K)
+            out = t.empty(M, N, dtype=t.float16, device=device)
+            nb = B.sqap_quantize_linear_workspace_bytes(M, N, K)
+            wsp = t.empty(nb, dtype=t.uint8, device=device)
+            sc_ptr = wsp.data_ptr() + B.sqap_workspace_bytes(M, N, K)
+            B.sqap_quantize_linear(x, M, K, None, 0, ws[0][0], ws[0][1], out, N, B.SQAP_FP16, 0, wsp, nb)
+            us = graph_time_us(t, lambda i: B.sqap_w4a4_linear(wsp, sc_ptr, M, ws[i % n][0], ws[i % n][1], out, N,
+                                                               B.SQAP_FP16, B.SQAP_L_REUSE_EXPANDED, wsp, nb),
+                               reps=max(n, 8))
+            ops = 2.0 * M * N * K * (2 if sw else 1)
+            byts = wbytes + M * K + 2 * M * N
+            if M >= 512:
+                add("w4a4_linear GEMM " + nm, f"M={M} N={N} K={K}", "tensor", ops, us)
+            else:
+                add("w4a4_linear GEMM " + nm, f"M={M} N={N} K={K}", "hbm", byts, us,
+                    note=f"{ops / (us * 1e-6) / 1e12:.0f} TOP/s = {ops / (us * 1e-6) / 1e12 / tpk:.2f} of tensor peak")
+            del x, out, wsp
+        for a, b in ws:
+            a.close()
+            if b:
+                b.close()
+    return rows
+
+
+def run_detail(args):
+    import torch
+    from paper_2509_09090_b200 import binding as B
+    torch.cuda.set_device(0)
+    dev = torch.device("cuda", 0)
+    peaks = measured_peaks()
+    rows = kernel_table(torch, B, peaks, dev)
+    torch.cuda.synchronize()
+    assert B.sqap_device_status() == B.SQAP_OK
+    print(json.dumps({"kernels": rows, "peaks": {"hbm_gbs": peaks["hbm_gbs"], "int8_tops": 2 * peaks["bf16"],
+                                                  "source": peaks["source"]}}))
+
+
 def run_single_kernel(args):
     """Profiling aid: a few launches of one kernel of the path on a small, larger-than-L2 case
     (what `ncu -k ... -c 3` captures). Prints nothing that counts as a bench value."""
@@ -446,10 +586,14 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--detail", action="store_true",
+                    help="time every kernel of the path alone at the workload's shapes (one JSON table, no bench line)")
     ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "quantize", "prune"],
                     help="profiling aid: launch only this kernel --steps times (no bench line)")
     args = ap.parse_args()
-    if args.kernel:
+    if args.detail:
+        run_detail(args)
+    elif args.kernel:
         run_single_kernel(args)
     elif args.impl == "reference":
         run_reference(args)

@@ -121,6 +121,25 @@ sqap_status sqap_w4a4_linear(const uint8_t* q_packed, const float* act_scales, i
                              void* workspace, size_t workspace_bytes, void* stream);
 
 /*
+ * Quantizer and linear as one call: what a W4A4 layer does with an fp16 activation ("4-bit activations" then
+ * Q = W_q^T X, Section 3.3; Eq. 6 when SQAP_Q_ROTATE is set). The result is exactly that of
+ *   sqap_quantize_act(x, M, K = w's K, ldx, row_index, qflags, q, s) ; sqap_w4a4_linear(q, s, M, w, w_up, out, ...)
+ * but the codes go straight from the quantizer's registers into the form the GEMM reads, so the nibble-packed
+ * intermediate is never written or re-read (3 bytes of HBM traffic per activation element instead of 4, one
+ * launch fewer). Arguments as in those two calls; lflags may hold a SQAP_L_FORCE_* flag (REUSE_EXPANDED is
+ * rejected). workspace: device scratch of at least sqap_quantize_linear_workspace_bytes(M, N, K) bytes,
+ * 256-byte aligned; afterwards it holds the expanded codes of these activations, so further weight matrices
+ * that take the SAME activations can follow with sqap_w4a4_linear(..., SQAP_L_REUSE_EXPANDED, workspace, ...)
+ * and act_scales = (const float*)((char*)workspace + sqap_workspace_bytes(M, N, K, 0)).
+ * Errors: those of the two calls.
+ */
+size_t sqap_quantize_linear_workspace_bytes(int M, int N, int K);
+sqap_status sqap_quantize_linear(const void* x, int M, int64_t ldx, const int32_t* row_index, uint32_t qflags,
+                                 const sqap_weights* w, const sqap_weights* w_up, void* out, int64_t ldo,
+                                 int out_dtype, uint32_t lflags, void* workspace, size_t workspace_bytes,
+                                 void* stream);
+
+/*
  * The same linear for callers that must not allocate. (The paper has no counterpart: this entry point
  * exists only for the sake of such callers.)
  *

@@ -21,6 +21,7 @@ SQAP_L_FORCE_SIMT, SQAP_L_FORCE_TCGEN05, SQAP_L_FORCE_GEMV, SQAP_L_REUSE_EXPANDE
 
 EXPORTS = ("sqap_pack_weights", "sqap_free_weights", "sqap_weights_info", "sqap_unpack_weights",
            "sqap_quantize_act", "sqap_workspace_bytes", "sqap_w4a4_linear", "sqap_w4a4_linear_static",
+           "sqap_quantize_linear", "sqap_quantize_linear_workspace_bytes",
            "sqap_prune_tokens",
            "sqap_project_center", "sqap_device_status", "sqap_last_cuda_error", "sqap_status_string",
            "sqap_kernel_launch_count")
@@ -62,6 +63,9 @@ def lib() -> ctypes.CDLL:
     L.sqap_workspace_bytes.restype = sz
     L.sqap_w4a4_linear.argtypes = [vp, vp, i32, vp, vp, vp, i64, i32, u32, vp, sz, vp]
     L.sqap_w4a4_linear_static.argtypes = [vp, vp, i32, vp, vp, vp, i64, i32, u32, vp]
+    L.sqap_quantize_linear_workspace_bytes.argtypes = [i32, i32, i32]
+    L.sqap_quantize_linear_workspace_bytes.restype = sz
+    L.sqap_quantize_linear.argtypes = [vp, i32, i64, vp, u32, vp, vp, vp, i64, i32, u32, vp, sz, vp]
     L.sqap_prune_tokens.argtypes = [ctypes.POINTER(PruneParams), vp, vp, vp, i64, i32, vp, i64, i32, vp, vp, vp]
     L.sqap_project_center.argtypes = [ctypes.POINTER(ctypes.c_double)] * 3 + [ctypes.c_double, ctypes.c_double,
                                                                               ctypes.POINTER(ctypes.c_int32),
@@ -162,6 +166,18 @@ def sqap_w4a4_linear(q_packed, act_scales, M: int, w: Weights, w_up, out, ldo: i
     _check(lib().sqap_w4a4_linear(_ptr(q_packed), _ptr(act_scales), M, w.handle, w_up.handle if w_up else None,
                                   _ptr(out), ldo, out_dtype, flags, _ptr(workspace), workspace_bytes,
                                   _stream(stream)), "sqap_w4a4_linear")
+
+
+def sqap_quantize_linear_workspace_bytes(M: int, N: int, K: int) -> int:
+    return int(lib().sqap_quantize_linear_workspace_bytes(M, N, K))
+
+
+def sqap_quantize_linear(x, M: int, ldx: int, row_index, qflags: int, w: Weights, w_up, out, ldo: int, out_dtype: int,
+                         lflags: int, workspace, workspace_bytes: int, stream=None):
+    """Quantizer and linear as one call (fp16 rows in, fp16/bf16 rows out); see include/sqap.h."""
+    _check(lib().sqap_quantize_linear(_ptr(x), M, ldx, _ptr(row_index), qflags, w.handle,
+                                      w_up.handle if w_up else None, _ptr(out), ldo, out_dtype, lflags,
+                                      _ptr(workspace), workspace_bytes, _stream(stream)), "sqap_quantize_linear")
 
 
 def sqap_w4a4_linear_static(q_packed, act_scales, M: int, w: Weights, w_up, out, ldo: int, out_dtype: int, flags: int,

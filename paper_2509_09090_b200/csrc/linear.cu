@@ -1,6 +1,7 @@
 // W4A4 linear: dispatcher, the activation expand pass, the CUDA-core GEMM (any shape) and the
 // weight-streaming kernel for very few rows. The tensor-core kernel lives in linear_tc.cu.
 #include "linear.cuh"
+#include "quantize.cuh"
 
 namespace sqap {
 
@@ -246,36 +247,30 @@ static size_t round256(size_t v) { return (v + 255) / 256 * 256; }
 
 }  // namespace sqap
 
-extern "C" {
+namespace sqap {
 
-size_t sqap_workspace_bytes(int M, int N, int K, uint32_t flags) {
-    (void)N;
-    (void)flags;
-    if (M <= 0 || K <= 0) return 256;
-    return sqap::round256(static_cast<size_t>(M) * K) + sqap::round256(sizeof(int32_t) * static_cast<size_t>(M));
-}
+enum LinearPath { PATH_SIMT, PATH_TC, PATH_GEMV };
 
-sqap_status sqap_w4a4_linear(const uint8_t* q_packed, const float* act_scales, int M, const sqap_weights* w,
-                             const sqap_weights* w_up, void* out, int64_t ldo, int out_dtype, uint32_t flags,
-                             void* workspace, size_t workspace_bytes, void* stream) {
-    using namespace sqap;
+// Argument rules shared by the entry points that run a linear (everything except the activation side).
+static sqap_status check_linear_args(int M, const sqap_weights* w, const sqap_weights* w_up, const void* out,
+                                     int64_t ldo, int out_dtype, uint32_t flags, uint32_t allowed_flags) {
     if (M < 0 || !w) return SQAP_ERR_INVALID;
     if (out_dtype != SQAP_FP16 && out_dtype != SQAP_BF16 && out_dtype != SQAP_I32) return SQAP_ERR_INVALID;
-    if (flags & ~(SQAP_L_FORCE_SIMT | SQAP_L_FORCE_TCGEN05 | SQAP_L_FORCE_GEMV | SQAP_L_REUSE_EXPANDED))
-        return SQAP_ERR_INVALID;
+    if (flags & ~allowed_flags) return SQAP_ERR_INVALID;
     const uint32_t force = flags & (SQAP_L_FORCE_SIMT | SQAP_L_FORCE_TCGEN05 | SQAP_L_FORCE_GEMV);
     if ((force & (force - 1)) != 0) return SQAP_ERR_INVALID;  // at most one forced kernel
     if (w_up && (w_up->N != w->N || w_up->K != w->K || w_up->half != w->half)) return SQAP_ERR_INVALID;
     if (w_up && out_dtype == SQAP_I32) return SQAP_ERR_INVALID;
     if (ldo < w->N) return SQAP_ERR_INVALID;
     if (M == 0) return SQAP_OK;
-    if (!q_packed || !act_scales || !out || !workspace) return SQAP_ERR_INVALID;
+    if (!out) return SQAP_ERR_INVALID;
     const int esz = out_dtype == SQAP_I32 ? 4 : 2;
-    if (!aligned16(q_packed) || !aligned16(out) || (ldo * esz) % 16 != 0) return SQAP_ERR_ALIGN;
-    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQAP_ERR_ALIGN;
-    if (workspace_bytes < sqap_workspace_bytes(M, w->N, w->K, flags)) return SQAP_ERR_NOMEM;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    if (!aligned16(out) || (ldo * esz) % 16 != 0) return SQAP_ERR_ALIGN;
+    return SQAP_OK;
+}
 
+static LinearArgs make_args(void* workspace, const float* act_scales, int M, const sqap_weights* w,
+                            const sqap_weights* w_up, void* out, int64_t ldo, int out_dtype) {
     LinearArgs a;
     a.x8 = static_cast<int8_t*>(workspace);
     a.bias_sum = reinterpret_cast<int32_t*>(static_cast<uint8_t*>(workspace) + round256(static_cast<size_t>(M) * w->K));
@@ -291,20 +286,69 @@ sqap_status sqap_w4a4_linear(const uint8_t* q_packed, const float* act_scales, i
     a.out = out;
     a.ldo = ldo;
     a.out_dtype = out_dtype;
+    return a;
+}
 
-    enum { SIMT, TC, GEMV } path;
-    if (flags & SQAP_L_FORCE_SIMT) path = SIMT;
+static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* path) {
+    if (flags & SQAP_L_FORCE_SIMT) *path = PATH_SIMT;
     else if (flags & SQAP_L_FORCE_GEMV) {
-        if (M > 8) return SQAP_ERR_UNSUPPORTED;
-        path = GEMV;
+        if (a.M > 8) return SQAP_ERR_UNSUPPORTED;
+        *path = PATH_GEMV;
     } else if (flags & SQAP_L_FORCE_TCGEN05) {
         if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
-        path = TC;
+        *path = PATH_TC;
     } else {
-        path = M <= 8 ? GEMV : (tcgen05_supports(a) ? TC : SIMT);
+        *path = a.M <= 8 ? PATH_GEMV : (tcgen05_supports(a) ? PATH_TC : PATH_SIMT);
     }
+    return SQAP_OK;
+}
 
-    sqap_status st = SQAP_OK;
+static sqap_status run_gemm(const LinearArgs& a, LinearPath path, cudaStream_t s) {
+    if (path == PATH_TC) return launch_linear_tcgen05(a, s);
+    if (path == PATH_GEMV) {
+        if (a.M == 1) launch_gemv<1>(a, s);
+        else if (a.M == 2) launch_gemv<2>(a, s);
+        else if (a.M <= 4) launch_gemv<4>(a, s);
+        else launch_gemv<8>(a, s);
+    } else {
+        dim3 grid((a.N + ST_N - 1) / ST_N, (a.M + ST_M - 1) / ST_M);
+        if (a.w_up) w4a4_simt_kernel<true><<<grid, 128, 0, s>>>(a);
+        else w4a4_simt_kernel<false><<<grid, 128, 0, s>>>(a);
+    }
+    count_launch();
+    return check_launch();
+}
+
+}  // namespace sqap
+
+extern "C" {
+
+size_t sqap_workspace_bytes(int M, int N, int K, uint32_t flags) {
+    (void)N;
+    (void)flags;
+    if (M <= 0 || K <= 0) return 256;
+    return sqap::round256(static_cast<size_t>(M) * K) + sqap::round256(sizeof(int32_t) * static_cast<size_t>(M));
+}
+
+sqap_status sqap_w4a4_linear(const uint8_t* q_packed, const float* act_scales, int M, const sqap_weights* w,
+                             const sqap_weights* w_up, void* out, int64_t ldo, int out_dtype, uint32_t flags,
+                             void* workspace, size_t workspace_bytes, void* stream) {
+    using namespace sqap;
+    sqap_status st = check_linear_args(M, w, w_up, out, ldo, out_dtype, flags,
+                                       SQAP_L_FORCE_SIMT | SQAP_L_FORCE_TCGEN05 | SQAP_L_FORCE_GEMV |
+                                           SQAP_L_REUSE_EXPANDED);
+    if (st != SQAP_OK || M == 0) return st;
+    if (!q_packed || !act_scales || !workspace) return SQAP_ERR_INVALID;
+    if (!aligned16(q_packed)) return SQAP_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQAP_ERR_ALIGN;
+    if (workspace_bytes < sqap_workspace_bytes(M, w->N, w->K, flags)) return SQAP_ERR_NOMEM;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    const LinearArgs a = make_args(workspace, act_scales, M, w, w_up, out, ldo, out_dtype);
+    LinearPath path;
+    st = pick_path(a, flags, &path);
+    if (st != SQAP_OK) return st;
+
     if (!(flags & SQAP_L_REUSE_EXPANDED)) {
         expand_act_kernel<<<M, 128, 0, s>>>(q_packed, a.K, a.half, const_cast<int8_t*>(a.x8),
                                             const_cast<int32_t*>(a.bias_sum));
@@ -312,20 +356,38 @@ sqap_status sqap_w4a4_linear(const uint8_t* q_packed, const float* act_scales, i
         st = check_launch();
         if (st != SQAP_OK) return st;
     }
+    return run_gemm(a, path, s);
+}
 
-    if (path == TC) return launch_linear_tcgen05(a, s);
-    if (path == GEMV) {
-        if (M == 1) launch_gemv<1>(a, s);
-        else if (M == 2) launch_gemv<2>(a, s);
-        else if (M <= 4) launch_gemv<4>(a, s);
-        else launch_gemv<8>(a, s);
-    } else {
-        dim3 grid((a.N + ST_N - 1) / ST_N, (M + ST_M - 1) / ST_M);
-        if (a.w_up) w4a4_simt_kernel<true><<<grid, 128, 0, s>>>(a);
-        else w4a4_simt_kernel<false><<<grid, 128, 0, s>>>(a);
-    }
-    count_launch();
-    return check_launch();
+size_t sqap_quantize_linear_workspace_bytes(int M, int N, int K) {
+    if (M <= 0 || K <= 0) return 256;
+    return sqap_workspace_bytes(M, N, K, 0) + sqap::round256(sizeof(float) * static_cast<size_t>(M));
+}
+
+sqap_status sqap_quantize_linear(const void* x, int M, int64_t ldx, const int32_t* row_index, uint32_t qflags,
+                                 const sqap_weights* w, const sqap_weights* w_up, void* out, int64_t ldo,
+                                 int out_dtype, uint32_t lflags, void* workspace, size_t workspace_bytes,
+                                 void* stream) {
+    using namespace sqap;
+    sqap_status st = check_linear_args(M, w, w_up, out, ldo, out_dtype, lflags,
+                                       SQAP_L_FORCE_SIMT | SQAP_L_FORCE_TCGEN05 | SQAP_L_FORCE_GEMV);
+    if (st != SQAP_OK) return st;
+    st = quantize_check_args(x, M, w->K, ldx, qflags);
+    if (st != SQAP_OK || M == 0) return st;
+    if (!workspace) return SQAP_ERR_INVALID;
+    if ((reinterpret_cast<uintptr_t>(workspace) & 255u) != 0) return SQAP_ERR_ALIGN;
+    if (workspace_bytes < sqap_quantize_linear_workspace_bytes(M, w->N, w->K)) return SQAP_ERR_NOMEM;
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+
+    float* scales = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + sqap_workspace_bytes(M, w->N, w->K, 0));
+    const LinearArgs a = make_args(workspace, scales, M, w, w_up, out, ldo, out_dtype);
+    LinearPath path;
+    st = pick_path(a, lflags, &path);
+    if (st != SQAP_OK) return st;
+    st = quantize_expanded(static_cast<const __half*>(x), M, a.K, ldx, row_index, qflags, a.half,
+                           const_cast<int8_t*>(a.x8), const_cast<int32_t*>(a.bias_sum), scales, s);
+    if (st != SQAP_OK) return st;
+    return run_gemm(a, path, s);
 }
 
 }  // extern "C"

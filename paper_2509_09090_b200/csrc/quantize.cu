@@ -1,16 +1,64 @@
 // Per-token symmetric INT4 activation quantizer with the optional Hadamard rotation of Eq. 6.
 //
-// HBM-bound: 2 bytes read and half a byte written per element. One CTA owns one row; the row
-// stays in registers between the max-abs reduction and the rounding pass, so global memory is
-// touched once. All fp32 steps use the explicitly rounded intrinsics, so no multiply-add is
-// fused and the result is defined bit for bit by the order of operations stated in sqap.h.
-#include "common.cuh"
+// HBM-bound for plain rows (2 bytes read, half a byte written per element); with the rotation the
+// 12 add/sub stages per element of K = 4096 put the fp32 pipes at about the same time as the memory
+// system. Global memory is touched once: a row stays in registers (and, for the rotation, shared
+// memory) between the max-abs reduction and the rounding pass. All fp32 steps use explicitly rounded,
+// unfused operations, so the result is defined bit for bit by the order of operations stated in sqap.h.
+//
+// Rounding without a float-to-int conversion: for |y| < 2^22, fl(y + 1.5 * 2^23) has an ulp of 1, so the
+// sum's low mantissa bits hold round_half_even(y) in two's complement. |v * inv| never exceeds 7 by more
+// than rounding error for finite inputs (|v| <= amax, inv = fl(7 / amax)), so the clamp of the definition
+// can never bind and is not evaluated; non-finite inputs give unspecified codes, as documented.
+//
+// Two output forms share every kernel (template parameter SINK):
+//   SINK_NIBBLES   the public layout of sqap_quantize_act (two codes per byte)
+//   SINK_EXPANDED  what the GEMM kernels multiply (linear.cuh): one int8 per code, codes that meet a low
+//                  weight nibble pre-multiplied by 16, plus the per-row sum of those codes. This skips the
+//                  expand pass when quantizer and linear run as one call (sqap_quantize_linear).
+#include "quantize.cuh"
 
 namespace sqap {
+
+constexpr int SINK_NIBBLES = 0, SINK_EXPANDED = 1;
+constexpr float MAGIC = 12582912.0f;   // 1.5 * 2^23: low byte of fl(y + MAGIC) = code as int8
+constexpr float MAGIC8 = 12582920.0f;  // MAGIC + 8:  low nibble of fl(y + MAGIC8) = code + 8 (0..15)
+
+struct QuantOut {
+    uint8_t* q;         // SINK_NIBBLES: [M][K/2]
+    int8_t* x8;         // SINK_EXPANDED: [M][K]
+    int32_t* bias_sum;  // SINK_EXPANDED: [M]
+    float* scales;      // [M]
+    int half;           // SINK_EXPANDED: half-block of the weight nibble pairing (64 or 16)
+};
+
+// ------------------------------------------------------------------------------- packed fp32 helpers
+__device__ __forceinline__ uint64_t pk(float lo, float hi) {
+    uint64_t r;
+    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
+    return r;
+}
+__device__ __forceinline__ void upk(uint64_t p, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p)); }
+__device__ __forceinline__ void upk_bits(uint64_t p, uint32_t& lo, uint32_t& hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(p)); }
+__device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("add.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+__device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
 
 __device__ __forceinline__ float warp_max(float v) {
 #pragma unroll
     for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
+    return v;
+}
+__device__ __forceinline__ int warp_sum(int v) {
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
     return v;
 }
 
@@ -26,98 +74,174 @@ __device__ __forceinline__ float block_max(float v, float* red) {
     __syncthreads();
     return r;
 }
-
-__device__ __forceinline__ int quant_code(float v, float inv) {
-    int q = __float2int_rn(__fmul_rn(v, inv));  // round half to even
-    return max(-8, min(7, q));
+__device__ __forceinline__ int block_sum(int v, int* red) {
+    v = warp_sum(v);
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31, nwarps = (blockDim.x + 31) >> 5;
+    if (nwarps == 1) return v;
+    if (lane == 0) red[warp] = v;
+    __syncthreads();
+    int r = (lane < nwarps) ? red[lane] : 0;
+    r = warp_sum(r);
+    __syncthreads();
+    return r;
 }
 
-// 8 fp32 values -> 8 two's-complement nibbles, value i in nibble i.
-__device__ __forceinline__ uint32_t pack8(const float* v, float inv) {
-    uint32_t w = 0;
-#pragma unroll
-    for (int i = 0; i < 8; ++i) w |= (static_cast<uint32_t>(quant_code(v[i], inv)) & 0xFu) << (4 * i);
-    return w;
-}
-
-__device__ __forceinline__ void unpack_half8(const uint4& u, float* f) {
-    const __half2* h = reinterpret_cast<const __half2*>(&u);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        float2 t = __half22float2(h[i]);
-        f[2 * i] = t.x;
-        f[2 * i + 1] = t.y;
-    }
-}
-
-// ---------------------------------------------------------------------------------------------
-// Plain (unrotated) rows. Thread t handles the 16-byte chunks t, t + T, t + 2T, ... of the row.
-// Up to MAX_IT chunks per thread are kept in registers; longer rows are re-read (L2 hit).
-constexpr int QUANT_MAX_IT = 8;
-
-__global__ void __launch_bounds__(256) quantize_rows_kernel(const __half* __restrict__ x, int K, int64_t ldx,
-                                                            const int32_t* __restrict__ row_index,
-                                                            uint8_t* __restrict__ q, float* __restrict__ scales) {
-    __shared__ float red[32];
-    const int row = blockIdx.x;
-    const int64_t src = row_index ? static_cast<int64_t>(row_index[row]) : static_cast<int64_t>(row);
-    const uint4* xr = reinterpret_cast<const uint4*>(x + src * ldx);
-    uint32_t* qr = reinterpret_cast<uint32_t*>(q + static_cast<int64_t>(row) * (K / 2));
-    const int chunks = K / 8;
-    const int T = blockDim.x;
-
-    uint4 cache[QUANT_MAX_IT];
-    float amax = 0.0f;
-#pragma unroll
-    for (int it = 0; it < QUANT_MAX_IT; ++it) {
-        const int c = it * T + threadIdx.x;
-        if (c < chunks) {
-            cache[it] = __ldg(xr + c);
-            float f[8];
-            unpack_half8(cache[it], f);
-#pragma unroll
-            for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(f[i]));
-        }
-    }
-    for (int c = QUANT_MAX_IT * T + threadIdx.x; c < chunks; c += T) {
-        float f[8];
-        unpack_half8(__ldg(xr + c), f);
-#pragma unroll
-        for (int i = 0; i < 8; ++i) amax = fmaxf(amax, fabsf(f[i]));
-    }
-    amax = block_max(amax, red);
-    float scale = 1.0f, inv = 0.0f;
+__device__ __forceinline__ void scale_of(float amax, float& scale, float& inv) {
+    scale = 1.0f;
+    inv = 0.0f;
     if (amax != 0.0f) {
         scale = __fdiv_rn(amax, 7.0f);
         inv = __fdiv_rn(7.0f, amax);
     }
-    if (threadIdx.x == 0) scales[row] = scale;
+}
+
+// Bits of fl(fl(v * inv) + magic) for a pair of values. The product must be rounded to fp32 before the sum
+// (a fused multiply-add rounds once and lands on the other side of a tie): scalar __fmul_rn / __fadd_rn are
+// never contracted, whereas a packed multiply followed by a packed add was seen to be.
+__device__ __forceinline__ void round_pair(uint64_t v, float inv, float magic, uint32_t& lo, uint32_t& hi) {
+    float a, b;
+    upk(v, a, b);
+    lo = __float_as_uint(__fadd_rn(__fmul_rn(a, inv), magic));
+    hi = __float_as_uint(__fadd_rn(__fmul_rn(b, inv), magic));
+}
+
+// Low bytes of four words -> one word.
+__device__ __forceinline__ uint32_t low_bytes(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3) {
+    return __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
+}
+// Two words of four bytes each holding code + 8 (0..15) -> eight two's-complement nibbles, value i in nibble i.
+__device__ __forceinline__ uint32_t nibbles_of(uint32_t w0, uint32_t w1) {
+    const uint32_t x0 = w0 | (w0 >> 4), x1 = w1 | (w1 >> 4);
+    return __byte_perm(x0, x1, 0x6420) ^ 0x88888888u;
+}
+// A word of four int8 codes -> the same codes times 16 (each still fits a byte).
+__device__ __forceinline__ uint32_t times16(uint32_t w) { return (w << 4) & 0xF0F0F0F0u; }
+
+// Eight consecutive values (k = 8c .. 8c+7 of the row) -> output. v as four packed pairs.
+template <int SINK>
+__device__ __forceinline__ void emit_chunk(const uint64_t* v, float inv, int c, const QuantOut& o, int64_t row,
+                                           int K, int& bias) {
+    const float magic = SINK == SINK_NIBBLES ? MAGIC8 : MAGIC;
+    uint32_t t[8];
 #pragma unroll
-    for (int it = 0; it < QUANT_MAX_IT; ++it) {
-        const int c = it * T + threadIdx.x;
-        if (c < chunks) {
-            float f[8];
-            unpack_half8(cache[it], f);
-            qr[c] = pack8(f, inv);
+    for (int i = 0; i < 4; ++i) round_pair(v[i], inv, magic, t[2 * i], t[2 * i + 1]);
+    const uint32_t w0 = low_bytes(t[0], t[1], t[2], t[3]), w1 = low_bytes(t[4], t[5], t[6], t[7]);
+    if (SINK == SINK_NIBBLES) {
+        reinterpret_cast<uint32_t*>(o.q + row * (K / 2))[c] = nibbles_of(w0, w1);
+    } else {
+        const bool low = ((8 * c) % (2 * o.half)) < o.half;
+        uint2 out = make_uint2(w0, w1);
+        if (low) {
+            bias = __dp4a(static_cast<int>(w0), 0x01010101, bias);
+            bias = __dp4a(static_cast<int>(w1), 0x01010101, bias);
+            out = make_uint2(times16(w0), times16(w1));
         }
+        reinterpret_cast<uint2*>(o.x8 + row * K)[c] = out;
     }
-    for (int c = QUANT_MAX_IT * T + threadIdx.x; c < chunks; c += T) {
-        float f[8];
-        unpack_half8(__ldg(xr + c), f);
-        qr[c] = pack8(f, inv);
+}
+
+__device__ __forceinline__ void half8_to_pairs(const uint4& u, uint64_t* p) {
+    const __half2* h = reinterpret_cast<const __half2*>(&u);
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        const float2 f = __half22float2(h[i]);
+        p[i] = pk(f.x, f.y);
     }
 }
 
 // ---------------------------------------------------------------------------------------------
-// Rotated rows: fast Walsh-Hadamard transform, stages h = 1, 2, 4, ..., K/2 in that order, each
-// pair (j, j+h) -> (a+b, a-b). Thread t holds the E contiguous elements E*t .. E*t+E-1, so the
-// first log2(E) stages are register-local, the next (up to 5) are warp shuffles, and the rest
-// go through shared memory. T = K / E threads.
-template <int E>
+// Plain (unrotated) rows. G threads own a row (256 / G rows per CTA); thread u of a row handles the 16-byte
+// chunks u, u + G, ... of it, up to QUANT_NIT of them held in registers (128 bytes in flight per thread);
+// longer rows are re-read in the second pass (L2 hit). The max-abs runs on the fp16 values themselves
+// (a maximum needs no widening).
+constexpr int QUANT_NIT = 8;
+constexpr int QUANT_THREADS = 256;
+
+template <int SINK, int G>
+__global__ void __launch_bounds__(QUANT_THREADS) quantize_rows_kernel(const __half* __restrict__ x, int M, int K,
+                                                                      int64_t ldx,
+                                                                      const int32_t* __restrict__ row_index,
+                                                                      QuantOut o) {
+    constexpr int ROWS = QUANT_THREADS / G, WARPS = G / 32;
+    __shared__ float red_f[ROWS][WARPS];
+    __shared__ int red_i[ROWS][WARPS];
+    const int g = threadIdx.x / G, u = threadIdx.x % G;
+    const int row = blockIdx.x * ROWS + g;
+    const bool row_ok = row < M;
+    const int64_t src = row_ok ? (row_index ? static_cast<int64_t>(row_index[row]) : static_cast<int64_t>(row)) : 0;
+    const uint4* xr = reinterpret_cast<const uint4*>(x + src * ldx);
+    const int chunks = row_ok ? K / 8 : 0;
+
+    uint4 cache[QUANT_NIT];
+    __half2 m2 = __float2half2_rn(0.0f);
+    auto absmax = [&](const uint4& v) {
+        const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+        for (int i = 0; i < 4; ++i) m2 = __hmax2(m2, __habs2(h[i]));
+    };
+#pragma unroll
+    for (int it = 0; it < QUANT_NIT; ++it) {
+        const int c = it * G + u;
+        if (c < chunks) cache[it] = __ldg(xr + c);
+    }
+#pragma unroll
+    for (int it = 0; it < QUANT_NIT; ++it)
+        if (it * G + u < chunks) absmax(cache[it]);
+    for (int c = QUANT_NIT * G + u; c < chunks; c += G) absmax(__ldg(xr + c));
+    float amax = warp_max(fmaxf(__low2float(m2), __high2float(m2)));
+    if (WARPS > 1) {
+        if ((u & 31) == 0) red_f[g][u >> 5] = amax;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < WARPS; ++w) amax = fmaxf(amax, red_f[g][w]);
+    }
+    float scale, inv;
+    scale_of(amax, scale, inv);
+    if (u == 0 && row_ok) o.scales[row] = scale;
+    int bias = 0;
+#pragma unroll
+    for (int it = 0; it < QUANT_NIT; ++it) {
+        const int c = it * G + u;
+        if (c < chunks) {
+            uint64_t p[4];
+            half8_to_pairs(cache[it], p);
+            emit_chunk<SINK>(p, inv, c, o, row, K, bias);
+        }
+    }
+    for (int c = QUANT_NIT * G + u; c < chunks; c += G) {
+        uint64_t p[4];
+        half8_to_pairs(__ldg(xr + c), p);
+        emit_chunk<SINK>(p, inv, c, o, row, K, bias);
+    }
+    if (SINK == SINK_EXPANDED) {
+        bias = warp_sum(bias);
+        if (WARPS > 1) {
+            if ((u & 31) == 0) red_i[g][u >> 5] = bias;
+            __syncthreads();
+            bias = 0;
+#pragma unroll
+            for (int w = 0; w < WARPS; ++w) bias += red_i[g][w];
+        }
+        if (u == 0 && row_ok) o.bias_sum[row] = bias;
+    }
+}
+
+template <int SINK, int G>
+static void launch_plain(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, const QuantOut& o,
+                         cudaStream_t s) {
+    constexpr int ROWS = QUANT_THREADS / G;
+    quantize_rows_kernel<SINK, G><<<(M + ROWS - 1) / ROWS, QUANT_THREADS, 0, s>>>(x, M, K, ldx, row_index, o);
+}
+
+// ---------------------------------------------------------------------------------------------
+// Rotated rows, any power-of-two K: fast Walsh-Hadamard transform, stages h = 1, 2, 4, ..., K/2 in that
+// order, each pair (j, j+h) -> (a+b, a-b). Thread t holds the E contiguous elements E*t .. E*t+E-1, so
+// the first log2(E) stages are register-local, the next (up to 5) are warp shuffles, and the rest go
+// through shared memory. T = K / E threads.
+template <int E, int SINK>
 __global__ void __launch_bounds__(1024) quantize_rows_rotate_kernel(const __half* __restrict__ x, int K, int64_t ldx,
                                                                     const int32_t* __restrict__ row_index,
-                                                                    float norm, uint8_t* __restrict__ q,
-                                                                    float* __restrict__ scales) {
+                                                                    float norm, QuantOut o) {
     extern __shared__ float sm[];  // K floats when K/E > 32, plus 32 for the reduction
     float* red = sm;
     float* buf = sm + 32;
@@ -131,11 +255,20 @@ __global__ void __launch_bounds__(1024) quantize_rows_rotate_kernel(const __half
     float v[E];
     if constexpr (E >= 8) {
 #pragma unroll
-        for (int c = 0; c < E / 8; ++c) unpack_half8(__ldg(reinterpret_cast<const uint4*>(xr) + c), v + 8 * c);
+        for (int c = 0; c < E / 8; ++c) {
+            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(xr) + c);
+            const __half2* h = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 f = __half22float2(h[i]);
+                v[8 * c + 2 * i] = f.x;
+                v[8 * c + 2 * i + 1] = f.y;
+            }
+        }
     } else {
 #pragma unroll
         for (int i = 0; i < E; i += 2) {
-            float2 f = __half22float2(*reinterpret_cast<const __half2*>(xr + i));
+            const float2 f = __half22float2(*reinterpret_cast<const __half2*>(xr + i));
             v[i] = f.x;
             v[i + 1] = f.y;
         }
@@ -182,39 +315,273 @@ __global__ void __launch_bounds__(1024) quantize_rows_rotate_kernel(const __half
         amax = fmaxf(amax, fabsf(v[j]));
     }
     amax = block_max(amax, red);
-    float scale = 1.0f, inv = 0.0f;
-    if (amax != 0.0f) {
-        scale = __fdiv_rn(amax, 7.0f);
-        inv = __fdiv_rn(7.0f, amax);
-    }
-    if (t == 0) scales[row] = scale;
-    uint8_t* qr = q + static_cast<int64_t>(row) * (K / 2) + static_cast<int64_t>(t) * (E / 2);
+    float scale, inv;
+    scale_of(amax, scale, inv);
+    if (t == 0) o.scales[row] = scale;
+    int bias = 0;
     if constexpr (E >= 8) {
-        uint32_t w[E / 8];
 #pragma unroll
-        for (int c = 0; c < E / 8; ++c) w[c] = pack8(v + 8 * c, inv);
-        if constexpr (E == 16) {
-            *reinterpret_cast<uint2*>(qr) = make_uint2(w[0], w[1]);
-        } else {
-            *reinterpret_cast<uint32_t*>(qr) = w[0];
+        for (int c = 0; c < E / 8; ++c) {
+            uint64_t p[4];
+#pragma unroll
+            for (int i = 0; i < 4; ++i) p[i] = pk(v[8 * c + 2 * i], v[8 * c + 2 * i + 1]);
+            emit_chunk<SINK>(p, inv, t * (E / 8) + c, o, row, K, bias);
         }
     } else {
+        // short rows (K = 64, 128): E = 2 or 4 values per thread, written bytewise
+        uint32_t code[E];
 #pragma unroll
-        for (int i = 0; i < E; i += 2)
-            qr[i / 2] = static_cast<uint8_t>((quant_code(v[i], inv) & 0xF) | ((quant_code(v[i + 1], inv) & 0xF) << 4));
+        for (int i = 0; i < E; ++i) code[i] = __float_as_uint(__fadd_rn(__fmul_rn(v[i], inv), MAGIC));
+        if (SINK == SINK_NIBBLES) {
+            uint8_t* qr = o.q + static_cast<int64_t>(row) * (K / 2) + static_cast<int64_t>(t) * (E / 2);
+#pragma unroll
+            for (int i = 0; i < E; i += 2) qr[i / 2] = static_cast<uint8_t>((code[i] & 0xFu) | ((code[i + 1] & 0xFu) << 4));
+        } else {
+            int8_t* xo = o.x8 + static_cast<int64_t>(row) * K + static_cast<int64_t>(t) * E;
+            const bool low = ((t * E) % (2 * o.half)) < o.half;  // E divides the half-block: uniform per thread
+#pragma unroll
+            for (int i = 0; i < E; ++i) {
+                const int qv = static_cast<int8_t>(code[i] & 0xFFu);
+                xo[i] = static_cast<int8_t>(low ? qv * 16 : qv);
+                if (low) bias += qv;
+            }
+        }
+    }
+    if (SINK == SINK_EXPANDED) {
+        bias = block_sum(bias, reinterpret_cast<int*>(red));
+        if (t == 0) o.bias_sum[row] = bias;
     }
 }
 
-template <int E>
-static void launch_rotate(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, uint8_t* q,
-                          float* scales, cudaStream_t s) {
+// ---------------------------------------------------------------------------------------------
+// Rotated rows of K = 4096, the hidden size of the backbone. 64 threads own a row (4 rows per CTA) and each
+// holds 64 values as 32 packed pairs (2i, 2i+1): the stage inside a pair is scalar, the other five of a pass
+// are packed add/sub on independent pairs. Pass A covers index bits 0-5 (h = 1..32) on 64 contiguous values;
+// one transpose through shared memory (128-bit stores, swizzled so that neither side has a bank conflict)
+// brings bits 6-11 into registers for pass B (h = 64..2048). The normalisation 1/sqrt(4096) = 2^-6 is exact,
+// so it is folded into the scale instead of multiplying every element: fl(v * 2^-6) * fl(7 / (amax * 2^-6))
+// and v * (fl(7 / (amax * 2^-6)) * 2^-6) are the same real product, rounded once.
+// The codes return through shared memory as bytes, so that the row is written out in order.
+constexpr int R4K = 4096, R4K_ROWS = 4, R4K_THREADS = 64 * R4K_ROWS;
+constexpr int R4K_SMEM = R4K_ROWS * R4K * 4 + R4K_THREADS * 128;  // transpose buffers + staging
+
+__device__ __forceinline__ void fwht64_pairs(uint64_t* P) {
+    // stage on bit 0: inside each pair
+#pragma unroll
+    for (int i = 0; i < 32; ++i) {
+        float a, b;
+        upk(P[i], a, b);
+        P[i] = pk(__fadd_rn(a, b), __fsub_rn(a, b));
+    }
+    // stages on bits 1-5: pair i with pair i + h/2
+#pragma unroll
+    for (int hp = 1; hp < 32; hp <<= 1) {
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            if ((i & hp) == 0) {
+                const uint64_t a = P[i], b = P[i + hp];
+                P[i] = add2(a, b);
+                P[i + hp] = sub2(a, b);
+            }
+        }
+    }
+}
+
+__device__ __forceinline__ void cp_async16(uint32_t dst_smem, const void* src) {
+    asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst_smem), "l"(src) : "memory");
+}
+__device__ __forceinline__ void cp_async_commit() { asm volatile("cp.async.commit_group;" ::: "memory"); }
+__device__ __forceinline__ void cp_async_wait_all() { asm volatile("cp.async.wait_group 0;" ::: "memory"); }
+// Barrier among the 64 threads of one row group (ids 1..4; id 0 is __syncthreads).
+__device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, 64;" ::"r"(g + 1) : "memory"); }
+
+// Persistent: a CTA walks rows blockIdx.x*4 + g, + 4*gridDim.x, ... . Each thread stages its own 128 input bytes
+// of the NEXT row with cp.async while the current row is transformed, so the HBM latency is off the critical path;
+// the staging slots are private to a thread (it alone writes and reads them), so they need no barrier.
+template <int SINK>
+__global__ void __launch_bounds__(R4K_THREADS, 2) quantize_rotate4096_kernel(const __half* __restrict__ x, int M,
+                                                                              int64_t ldx,
+                                                                              const int32_t* __restrict__ row_index,
+                                                                              QuantOut o) {
+    extern __shared__ __align__(16) uint8_t smem_raw[];
+    __shared__ float red_f[R4K_ROWS][2];
+    __shared__ int red_i[R4K_ROWS][2];
+    const int g = threadIdx.x >> 6, u = threadIdx.x & 63;  // row group, thread within the row
+    float* buf = reinterpret_cast<float*>(smem_raw) + g * R4K;
+    uint8_t* bytes = reinterpret_cast<uint8_t*>(buf);
+    uint8_t* stage = smem_raw + R4K_ROWS * R4K * 4 + (g * 64 + u) * 128;  // this thread's 8 chunks, swizzled by u
+    const uint32_t stage_u32 = static_cast<uint32_t>(__cvta_generic_to_shared(stage));
+    const int row_step = gridDim.x * R4K_ROWS;
+
+    auto prefetch = [&](int row) {
+        if (row < M) {
+            const int64_t src = row_index ? static_cast<int64_t>(row_index[row]) : static_cast<int64_t>(row);
+            const uint4* xr = reinterpret_cast<const uint4*>(x + src * ldx) + u * 8;
+#pragma unroll
+            for (int c = 0; c < 8; ++c) cp_async16(stage_u32 + ((c ^ (u & 7)) << 4), xr + c);
+        }
+        cp_async_commit();
+    };
+
+    int row = blockIdx.x * R4K_ROWS + g;
+    prefetch(row);
+    for (; row < M; row += row_step) {
+        uint64_t P[32];
+        cp_async_wait_all();
+#pragma unroll
+        for (int c = 0; c < 8; ++c)
+            half8_to_pairs(*reinterpret_cast<const uint4*>(stage + ((c ^ (u & 7)) << 4)), P + 4 * c);
+        prefetch(row + row_step);  // the values above are in registers: the slots are free again
+        fwht64_pairs(P);           // h = 1 .. 32
+
+        // transpose: value r of thread u -> float u*64 + (r ^ ((u & 7) << 2)); 16 bytes = values 4g4 .. 4g4+3
+#pragma unroll
+        for (int g4 = 0; g4 < 16; ++g4) {
+            uint32_t a0, a1, b0, b1;
+            upk_bits(P[2 * g4], a0, a1);
+            upk_bits(P[2 * g4 + 1], b0, b1);
+            *reinterpret_cast<uint4*>(buf + u * 64 + ((g4 ^ (u & 7)) << 2)) = make_uint4(a0, a1, b0, b1);
+        }
+        group_sync(g);
+        // thread u now takes value u of every thread r: element index r*64 + u
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            const int r0 = 2 * i, r1 = 2 * i + 1;
+            const float lo = buf[r0 * 64 + (u ^ ((r0 & 7) << 2))];
+            const float hi = buf[r1 * 64 + (u ^ ((r1 & 7) << 2))];
+            P[i] = pk(lo, hi);
+        }
+        fwht64_pairs(P);  // h = 64 .. 2048
+
+        float amax = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            float a, b;
+            upk(P[i], a, b);
+            amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+        }
+        amax = warp_max(amax);
+        if ((u & 31) == 0) red_f[g][u >> 5] = amax;
+        group_sync(g);  // also: every read of buf above is done before the bytes below overwrite it
+        amax = fmaxf(red_f[g][0], red_f[g][1]) * 0.015625f;  // exact
+        float scale, inv;
+        scale_of(amax, scale, inv);
+        if (u == 0) o.scales[row] = scale;
+        inv *= 0.015625f;  // exact
+        const float magic = SINK == SINK_NIBBLES ? MAGIC8 : MAGIC;
+#pragma unroll
+        for (int i = 0; i < 32; ++i) {
+            uint32_t t0, t1;
+            round_pair(P[i], inv, magic, t0, t1);
+            bytes[(2 * i) * 64 + u] = static_cast<uint8_t>(t0);
+            bytes[(2 * i + 1) * 64 + u] = static_cast<uint8_t>(t1);
+        }
+        group_sync(g);
+        // write-out: thread u takes the 16-code chunks u, u + 64, u + 128, u + 192 of the row
+        int bias = 0;
+#pragma unroll
+        for (int i = 0; i < 4; ++i) {
+            const int c = u + 64 * i;
+            const uint4 w = *reinterpret_cast<const uint4*>(bytes + 16 * c);
+            if (SINK == SINK_NIBBLES) {
+                reinterpret_cast<uint2*>(o.q + static_cast<int64_t>(row) * (R4K / 2))[c] =
+                    make_uint2(nibbles_of(w.x, w.y), nibbles_of(w.z, w.w));
+            } else {
+                uint4 out = w;
+                if ((c & 4) == 0) {  // codes 16c .. 16c+15 lie in the first 64 of their block of 128
+                    bias = __dp4a(static_cast<int>(w.x), 0x01010101, bias);
+                    bias = __dp4a(static_cast<int>(w.y), 0x01010101, bias);
+                    bias = __dp4a(static_cast<int>(w.z), 0x01010101, bias);
+                    bias = __dp4a(static_cast<int>(w.w), 0x01010101, bias);
+                    out = make_uint4(times16(w.x), times16(w.y), times16(w.z), times16(w.w));
+                }
+                reinterpret_cast<uint4*>(o.x8 + static_cast<int64_t>(row) * R4K)[c] = out;
+            }
+        }
+        if (SINK == SINK_EXPANDED) {
+            bias = warp_sum(bias);
+            if ((u & 31) == 0) red_i[g][u >> 5] = bias;
+        }
+        group_sync(g);  // bytes (and red_f / red_i) are read: the next row may overwrite them
+        if (SINK == SINK_EXPANDED && u == 0) o.bias_sum[row] = red_i[g][0] + red_i[g][1];
+    }
+    cp_async_wait_all();
+}
+
+static int num_sms() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+template <int E, int SINK>
+static void launch_rotate(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, const QuantOut& o,
+                          cudaStream_t s) {
     const int T = K / E;
     const float norm = static_cast<float>(1.0 / sqrt(static_cast<double>(K)));
     const size_t smem = (32 + (T > 32 ? static_cast<size_t>(K) : 0)) * sizeof(float);
     if (smem > 48 * 1024)
-        cudaFuncSetAttribute(quantize_rows_rotate_kernel<E>, cudaFuncAttributeMaxDynamicSharedMemorySize,
+        cudaFuncSetAttribute(quantize_rows_rotate_kernel<E, SINK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
                              static_cast<int>(smem));
-    quantize_rows_rotate_kernel<E><<<M, T, smem, s>>>(x, K, ldx, row_index, norm, q, scales);
+    quantize_rows_rotate_kernel<E, SINK><<<M, T, smem, s>>>(x, K, ldx, row_index, norm, o);
+}
+
+template <int SINK>
+static sqap_status launch_quantize(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, bool rotate,
+                                   const QuantOut& o, cudaStream_t s) {
+    if (rotate) {
+        if (K == R4K) {
+            static bool attr_set = false;  // per process; the attribute is per function and device-independent here
+            if (!attr_set) {
+                cudaError_t e = cudaFuncSetAttribute(quantize_rotate4096_kernel<SINK>,
+                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, R4K_SMEM);
+                if (e != cudaSuccess) {
+                    note_cuda_error(e);
+                    return SQAP_ERR_CUDA;
+                }
+                attr_set = true;
+            }
+            int ctas = (M + R4K_ROWS - 1) / R4K_ROWS;
+            const int resident = 2 * num_sms();
+            if (ctas > resident) ctas = resident;
+            quantize_rotate4096_kernel<SINK><<<ctas, R4K_THREADS, R4K_SMEM, s>>>(x, M, ldx, row_index, o);
+        }
+        // E elements per thread: 16 from K = 512 up (T = K/16 <= 1024), fewer for short rows so a full warp works
+        else if (K >= 512) launch_rotate<16, SINK>(x, M, K, ldx, row_index, o, s);
+        else if (K == 256) launch_rotate<8, SINK>(x, M, K, ldx, row_index, o, s);
+        else if (K == 128) launch_rotate<4, SINK>(x, M, K, ldx, row_index, o, s);
+        else launch_rotate<2, SINK>(x, M, K, ldx, row_index, o, s);
+    } else {
+        // the fewest threads per row that keep the whole row in registers (8 chunks of 8 values per thread)
+        const int chunks = K / 8;
+        if (chunks <= 32 * QUANT_NIT) launch_plain<SINK, 32>(x, M, K, ldx, row_index, o, s);
+        else if (chunks <= 64 * QUANT_NIT) launch_plain<SINK, 64>(x, M, K, ldx, row_index, o, s);
+        else if (chunks <= 128 * QUANT_NIT) launch_plain<SINK, 128>(x, M, K, ldx, row_index, o, s);
+        else launch_plain<SINK, 256>(x, M, K, ldx, row_index, o, s);
+    }
+    count_launch();
+    return check_launch();
+}
+
+sqap_status quantize_check_args(const void* x, int M, int K, int64_t ldx, uint32_t flags) {
+    if (M < 0 || K <= 0 || ldx < K) return SQAP_ERR_INVALID;
+    if (flags & ~SQAP_Q_ROTATE) return SQAP_ERR_INVALID;
+    if (M == 0) return SQAP_OK;
+    if (!x) return SQAP_ERR_INVALID;
+    if (K % 32 != 0 || ldx % 8 != 0 || !aligned16(x)) return SQAP_ERR_ALIGN;
+    if ((flags & SQAP_Q_ROTATE) && ((K & (K - 1)) != 0 || K < 64 || K > 16384)) return SQAP_ERR_UNSUPPORTED;
+    return SQAP_OK;
+}
+
+sqap_status quantize_expanded(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, uint32_t flags,
+                              int half, int8_t* x8, int32_t* bias_sum, float* scales, cudaStream_t s) {
+    QuantOut o{nullptr, x8, bias_sum, scales, half};
+    return launch_quantize<SINK_EXPANDED>(x, M, K, ldx, row_index, (flags & SQAP_Q_ROTATE) != 0, o, s);
 }
 
 }  // namespace sqap
@@ -222,26 +589,12 @@ static void launch_rotate(const __half* x, int M, int K, int64_t ldx, const int3
 extern "C" sqap_status sqap_quantize_act(const void* x, int M, int K, int64_t ldx, const int32_t* row_index,
                                          uint32_t flags, uint8_t* q_packed, float* scales, void* stream) {
     using namespace sqap;
-    if (M < 0 || K <= 0 || ldx < K) return SQAP_ERR_INVALID;
-    if (flags & ~SQAP_Q_ROTATE) return SQAP_ERR_INVALID;
-    if (M == 0) return SQAP_OK;
-    if (!x || !q_packed || !scales) return SQAP_ERR_INVALID;
-    if (K % 32 != 0 || ldx % 8 != 0 || !aligned16(x) || !aligned16(q_packed)) return SQAP_ERR_ALIGN;
+    const sqap_status st = quantize_check_args(x, M, K, ldx, flags);
+    if (st != SQAP_OK || M == 0) return st;
+    if (!q_packed || !scales) return SQAP_ERR_INVALID;
+    if (!aligned16(q_packed)) return SQAP_ERR_ALIGN;
     if (reinterpret_cast<uintptr_t>(scales) & 3u) return SQAP_ERR_ALIGN;
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const __half* xh = static_cast<const __half*>(x);
-    if (flags & SQAP_Q_ROTATE) {
-        if ((K & (K - 1)) != 0 || K < 64 || K > 16384) return SQAP_ERR_UNSUPPORTED;
-        // E elements per thread: 16 from K = 512 up (T = K/16 <= 1024), fewer for short rows so a full warp works
-        if (K >= 512) launch_rotate<16>(xh, M, K, ldx, row_index, q_packed, scales, s);
-        else if (K == 256) launch_rotate<8>(xh, M, K, ldx, row_index, q_packed, scales, s);
-        else if (K == 128) launch_rotate<4>(xh, M, K, ldx, row_index, q_packed, scales, s);
-        else launch_rotate<2>(xh, M, K, ldx, row_index, q_packed, scales, s);
-    } else {
-        int T = (K / 8 + 31) / 32 * 32;
-        if (T > 256) T = 256;
-        quantize_rows_kernel<<<M, T, 0, s>>>(xh, K, ldx, row_index, q_packed, scales);
-    }
-    count_launch();
-    return check_launch();
+    QuantOut o{q_packed, nullptr, nullptr, scales, 64};
+    return launch_quantize<SINK_NIBBLES>(static_cast<const __half*>(x), M, K, ldx, row_index,
+                                         (flags & SQAP_Q_ROTATE) != 0, o, static_cast<cudaStream_t>(stream));
 }

@@ -69,6 +69,33 @@ def linear(packed: np.ndarray, scales: np.ndarray, w: B.Weights, w_up=None, out_
     return o if out_dtype == B.SQAP_I32 else o.view(np.uint16)
 
 
+def quantize_linear(x_f16: np.ndarray, w: B.Weights, w_up=None, rotate: bool = False, row_index=None,
+                    out_dtype=B.SQAP_FP16, flags=0, col_offset: int = 0):
+    """The fused call on the columns [col_offset, col_offset + K) of x_f16; output as in linear()."""
+    xd = to_dev(np.ascontiguousarray(x_f16, dtype=np.float16))
+    rows, ld = x_f16.shape
+    ri = to_dev(np.asarray(row_index, np.int32)) if row_index is not None else None
+    M = len(row_index) if row_index is not None else rows
+    N = w.N
+    ldo = (N + 7) // 8 * 8
+    tdt = torch.int32 if out_dtype == B.SQAP_I32 else torch.int16
+    fill = 0x7B7B7B7B if out_dtype == B.SQAP_I32 else 0x7B7B
+    out = torch.full((M + 1, ldo), fill, dtype=tdt, device=DEV)
+    nbytes = B.sqap_quantize_linear_workspace_bytes(M, N, w.K)
+    ws = torch.empty(nbytes + 256, dtype=torch.uint8, device=DEV)
+    ws_ptr = (ws.data_ptr() + 255) // 256 * 256
+    B.sqap_quantize_linear(xd.data_ptr() + 2 * col_offset, M, ld, ri, B.SQAP_Q_ROTATE if rotate else 0, w, w_up, out,
+                           ldo, out_dtype, flags, ws_ptr, nbytes)
+    torch.cuda.synchronize()
+    assert B.sqap_device_status() == B.SQAP_OK
+    o = out.cpu().numpy()
+    assert (o[M] == (fill if out_dtype == B.SQAP_I32 else np.int16(fill))).all(), "wrote past the last row"
+    if ldo > N:
+        assert (o[:M, N:] == o[M, 0]).all(), "wrote past the row end"
+    o = o[:M, :N]
+    return o if out_dtype == B.SQAP_I32 else o.view(np.uint16)
+
+
 def prune(params: dict, scores: np.ndarray, centers=None, x_f16=None, out_rows: int = 0, K=None):
     """Returns (kept_idx [B, rows], n_kept [B], x_out [B, out_rows, K] bits or None)."""
     Bn, rows = params["batch"], params["rows"]

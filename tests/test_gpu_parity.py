@@ -50,6 +50,13 @@ def check_linear(x_f16, w_codes, w_scales, rotate=False, row_index=None, up=None
         out = G.linear(packed_g, s_g, w, w_up=wu, out_dtype=B.SQAP_BF16 if bf16 else B.SQAP_FP16, flags=flags)
         ok = G.within_tolerance(out, ref, bf16=bf16)
         assert ok.all(), f"{(~ok).sum()} outputs outside tolerance (flags={flags})"
+        # the fused quantize + linear call: same accumulators, and the same output bits as the two-call route
+        if up is None:
+            acc_f = G.quantize_linear(x_f16, w, rotate=rotate, row_index=row_index, out_dtype=B.SQAP_I32, flags=flags)
+            assert np.array_equal(acc_f, acc_o), f"fused call: int32 accumulators differ (flags={flags})"
+        out_f = G.quantize_linear(x_f16, w, w_up=wu, rotate=rotate, row_index=row_index,
+                                  out_dtype=B.SQAP_BF16 if bf16 else B.SQAP_FP16, flags=flags)
+        assert np.array_equal(out_f, out), f"fused call differs from quantize_act + w4a4_linear (flags={flags})"
     w.close()
     if wu:
         wu.close()
@@ -70,6 +77,31 @@ def test_quantizer_bit_exact(M, K, rotate):
     pg, sg = G.quantize(x, rotate=rotate)
     assert np.array_equal(pg, po)
     assert np.array_equal(sg, so)
+
+
+@pytest.mark.parametrize("K,rotate", [(512, False), (4096, False), (11008, False)])
+def test_quantizer_products_that_round_onto_a_tie(K, rotate):
+    """v = amax/2 gives v * fl(7/amax) = 3.5 * (1 + d), |d| <= 2^-24: for many amax the fp32 product rounds to
+    exactly 3.5 and the tie goes to 4, while a multiply fused with the next operation sees 3.5 - tiny and gives
+    3. The rows where that happens are found here in fp64; they catch a kernel that does not round the product."""
+    M = 64
+    x = (wl.activations(77, K, M, K, 0, 1.0) * np.float16(0.01)).astype(np.float16)
+    amax = (np.arange(M, dtype=np.float32) * 0.71875 + 40.0).astype(np.float16)
+    for r in range(M):
+        x[r, 5], x[r, K // 2 + 1], x[r, K - 2] = amax[r], amax[r] / np.float16(2), -amax[r] / np.float16(2)
+    po, so, codes = oracle.quantize_act(bits(x), rotate=rotate)
+    inv = np.float32(7.0) / amax.astype(np.float32)
+    exact = amax.astype(np.float64) / 2 * inv.astype(np.float64)          # 11 x 24 bits: exact in fp64
+    onto_tie_from_below = (exact.astype(np.float32) == np.float32(3.5)) & (exact < 3.5)
+    assert onto_tie_from_below.sum() >= 16
+    assert (codes[onto_tie_from_below, K // 2 + 1] == 4).all() and (codes[onto_tie_from_below, K - 2] == -4).all()
+    pg, sg = G.quantize(x, rotate=rotate)
+    assert np.array_equal(pg, po) and np.array_equal(sg, so)
+    wc, ws = wl.weight_codes(77, K, 8, K), wl.weight_scales(77, K, 8)
+    w = G.pack(wc, ws)
+    acc = G.quantize_linear(x, w, rotate=rotate, out_dtype=B.SQAP_I32)
+    assert np.array_equal(acc, oracle.gemm_i32(codes, wc))
+    w.close()
 
 
 def test_quantizer_row_index_stride_and_empty():
@@ -160,6 +192,20 @@ def test_linear_tcgen05_forced(M, N, K, swiglu):
     u = (wl.weight_codes(25, N + K + 1, N, K), wl.weight_scales(25, N + K + 1, N, mult=0.5)) if swiglu else None
     check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05])
     check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05], bf16=True)
+
+
+@pytest.mark.parametrize("K", [64, 128, 256, 512, 4096])
+def test_fused_quantize_linear_rotated_rows_and_row_index(K):
+    """The fused call with the Hadamard rotation at every supported row length class, reading its rows
+    through an index list (repeated and out-of-order rows), against the oracle."""
+    M, N = 37, 72
+    x = wl.activations(27, K, 50, K, max(1, K // 100), 30.0)
+    x[11] = 0
+    idx = [(7 * i + 3) % 50 for i in range(M - 1)] + [11]
+    wc = wl.weight_codes(27, N + K, N, K)
+    ws = wl.weight_scales(27, N + K, N)
+    check_linear(x, wc, ws, rotate=True, row_index=idx)
+    check_linear(x, wc, ws, rotate=False, row_index=idx)
 
 
 @pytest.mark.parametrize("M", [1, 2, 3, 5, 8])
