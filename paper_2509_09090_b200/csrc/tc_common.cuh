@@ -1,0 +1,225 @@
+// Pieces shared by the tcgen05 kernels of the W4A4 linear: PTX wrappers, the epilogue of one accumulator
+// tile, tensor-map creation.
+#pragma once
+
+#include <cuda.h>
+
+#include "linear.cuh"
+
+namespace sqap {
+namespace tc {
+
+constexpr long long WAIT_LIMIT_CLOCKS = 4000000000LL;  // ~2 s
+
+struct Args {
+    const int32_t* bias_sum;
+    const float* act_scales;
+    const __half* w_scales;
+    const __half* w_up_scales;
+    void* out;
+    int64_t ldo;
+    int M, N, K;
+    int BN;        // tokens per tile
+    int m_tiles, n_tiles;
+    int out_dtype;
+    int swiglu;    // 1: tile rows 2i / 2i+1 hold gate / up of output channel n0/2 + i
+    int* status;
+};
+
+// ------------------------------------------------------------------------------- PTX wrappers
+__device__ __forceinline__ uint32_t smem_u32(const void* p) { return static_cast<uint32_t>(__cvta_generic_to_shared(p)); }
+
+__device__ __forceinline__ void mbar_init(uint32_t bar, uint32_t count) {
+    asm volatile("mbarrier.init.shared::cta.b64 [%0], %1;" ::"r"(bar), "r"(count));
+}
+__device__ __forceinline__ void mbar_expect_tx(uint32_t bar, uint32_t bytes) {
+    asm volatile("mbarrier.arrive.expect_tx.shared::cta.b64 _, [%0], %1;" ::"r"(bar), "r"(bytes) : "memory");
+}
+__device__ __forceinline__ void mbar_arrive(uint32_t bar) {
+    asm volatile("mbarrier.arrive.shared::cta.b64 _, [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ bool mbar_try_wait(uint32_t bar, uint32_t parity) {
+    uint32_t ok;
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "mbarrier.try_wait.parity.shared::cta.b64 p, [%1], %2;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(ok)
+        : "r"(bar), "r"(parity)
+        : "memory");
+    return ok != 0;
+}
+// Bounded wait: false if the phase did not complete within WAIT_LIMIT_CLOCKS or another role gave up.
+__device__ __forceinline__ bool mbar_wait(uint32_t bar, uint32_t parity, volatile int* abort_flag) {
+    if (mbar_try_wait(bar, parity)) return true;
+    const long long t0 = clock64();
+    uint32_t spins = 0;
+    while (!mbar_try_wait(bar, parity)) {
+        if ((++spins & 0x3FFu) == 0) {
+            if (*abort_flag) return false;
+            if (clock64() - t0 > WAIT_LIMIT_CLOCKS) return false;
+        }
+    }
+    return true;
+}
+__device__ __forceinline__ void tma_load_2d(uint32_t dst, const CUtensorMap* map, int c0, int c1, uint32_t bar) {
+    asm volatile(
+        "cp.async.bulk.tensor.2d.shared::cluster.global.mbarrier::complete_tx::bytes [%0], [%1, {%2, %3}], [%4];"
+        ::"r"(dst), "l"(reinterpret_cast<uint64_t>(map)), "r"(c0), "r"(c1), "r"(bar)
+        : "memory");
+}
+__device__ __forceinline__ void fence_proxy_async() { asm volatile("fence.proxy.async.shared::cta;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_before() { asm volatile("tcgen05.fence::before_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_fence_after() { asm volatile("tcgen05.fence::after_thread_sync;" ::: "memory"); }
+__device__ __forceinline__ void tc_commit(uint32_t bar) {
+    asm volatile("tcgen05.commit.cta_group::1.mbarrier::arrive::one.shared::cluster.b64 [%0];" ::"r"(bar) : "memory");
+}
+__device__ __forceinline__ void tc_mma_i8(uint32_t d_tmem, uint64_t adesc, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], %1, %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "l"(adesc), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+__device__ __forceinline__ void tc_ld16(uint32_t taddr, uint32_t* r) {
+    asm volatile(
+        "tcgen05.ld.sync.aligned.32x32b.x16.b32 {%0, %1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15}, [%16];"
+        : "=r"(r[0]), "=r"(r[1]), "=r"(r[2]), "=r"(r[3]), "=r"(r[4]), "=r"(r[5]), "=r"(r[6]), "=r"(r[7]), "=r"(r[8]),
+          "=r"(r[9]), "=r"(r[10]), "=r"(r[11]), "=r"(r[12]), "=r"(r[13]), "=r"(r[14]), "=r"(r[15])
+        : "r"(taddr)
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_ld() { asm volatile("tcgen05.wait::ld.sync.aligned;" ::: "memory"); }
+
+// K-major, 128-byte-swizzled operand tile: rows 128 B apart, 8-row groups 1024 B apart.
+__device__ __forceinline__ uint64_t smem_desc_sw128(uint32_t addr) {
+    return static_cast<uint64_t>((addr >> 4) & 0x3FFFu) | (1ull << 16) | (64ull << 32) | (1ull << 46) | (2ull << 61);
+}
+
+__device__ __forceinline__ float silu_mul_fast(float g, float u) { return __fdividef(g, 1.0f + __expf(-g)) * u; }
+
+// Part of one finished accumulator tile -> global memory. The thread owns one TMEM lane (output channel n;
+// with SwiGLU the even lane of a pair holds the gate and the odd lane the up projection of channel n) and
+// walks the tokens [c_begin, c_end) of the tile 16 at a time; the per-token bias sums and scales of a chunk
+// are fetched by lanes 0-15 with one coalesced load each (one chunk ahead) and broadcast by shuffle.
+template <int OUT, bool SWIGLU>
+__device__ __forceinline__ void epilogue_tile(const Args& a, uint32_t taddr, int m0, int c_begin, int c_end, int n,
+                                              bool n_ok, float sw, int lane) {
+    constexpr int ESZ = OUT == SQAP_I32 ? 4 : 2;
+    const int ml = lane & 15;
+    const bool odd = (lane & 1) != 0;
+    const int64_t row_bytes = a.ldo * ESZ;
+    int mm = m0 + c_begin + ml;
+    int bs_next = mm < a.M ? (__ldg(a.bias_sum + mm) << 7) : 0;
+    float sx_next = mm < a.M ? __ldg(a.act_scales + mm) : 0.0f;
+    for (int c = c_begin; c < c_end; c += 16) {
+        uint32_t v[16];
+        tc_ld16(taddr + c, v);
+        const int bs_cur = bs_next;
+        const float sx_cur = sx_next;
+        mm = m0 + c + 16 + ml;
+        if (c + 16 < c_end) {
+            bs_next = mm < a.M ? (__ldg(a.bias_sum + mm) << 7) : 0;
+            sx_next = mm < a.M ? __ldg(a.act_scales + mm) : 0.0f;
+        }
+        tc_wait_ld();
+        const int valid = a.M - (m0 + c);  // tokens of this chunk that exist
+        uint8_t* optr = static_cast<uint8_t*>(a.out) + static_cast<int64_t>(m0 + c) * row_bytes + static_cast<int64_t>(n) * ESZ;
+        if (SWIGLU) {
+            // Columns are handled in pairs: the even lane finishes column j (needs the up value of its
+            // partner), the odd lane column j+1 (needs the gate value of its partner): one exchange per pair.
+#pragma unroll
+            for (int j = 0; j < 16; j += 2) {
+                const float y0 = __fmul_rn(__fmul_rn(static_cast<float>((static_cast<int>(v[j]) - __shfl_sync(0xffffffffu, bs_cur, j)) >> 4),
+                                                     __shfl_sync(0xffffffffu, sx_cur, j)), sw);
+                const float y1 = __fmul_rn(__fmul_rn(static_cast<float>((static_cast<int>(v[j + 1]) - __shfl_sync(0xffffffffu, bs_cur, j + 1)) >> 4),
+                                                     __shfl_sync(0xffffffffu, sx_cur, j + 1)), sw);
+                const float got = __shfl_xor_sync(0xffffffffu, odd ? y0 : y1, 1);
+                const float h = odd ? silu_mul_fast(got, y1) : silu_mul_fast(y0, got);
+                const int jj = odd ? j + 1 : j;
+                if (n_ok && jj < valid) {
+                    uint8_t* o = optr + jj * row_bytes;
+                    if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(h);
+                    else *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(h);
+                }
+            }
+        } else {
+#pragma unroll
+            for (int j = 0; j < 16; ++j) {
+                const int bs = __shfl_sync(0xffffffffu, bs_cur, j);
+                const float sx = __shfl_sync(0xffffffffu, sx_cur, j);
+                const int t = (static_cast<int>(v[j]) - bs) >> 4;
+                const float y = __fmul_rn(__fmul_rn(static_cast<float>(t), sx), sw);
+                if (n_ok && j < valid) {
+                    if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(optr) = __float2half_rn(y);
+                    else if (OUT == SQAP_BF16) *reinterpret_cast<__nv_bfloat16*>(optr) = __float2bfloat16_rn(y);
+                    else *reinterpret_cast<int32_t*>(optr) = t;
+                }
+                optr += row_bytes;
+            }
+        }
+    }
+}
+
+// ------------------------------------------------------------------------------- host side
+typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
+                                  const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
+                                  CUtensorMapSwizzle, CUtensorMapL2promotion, CUtensorMapFloatOOBfill);
+
+inline EncodeTiledFn encode_fn() {
+    static EncodeTiledFn fn = nullptr;
+    static bool tried = false;
+    if (!tried) {
+        tried = true;
+        void* p = nullptr;
+        cudaDriverEntryPointQueryResult q;
+        if (cudaGetDriverEntryPoint("cuTensorMapEncodeTiled", &p, cudaEnableDefault, &q) == cudaSuccess &&
+            q == cudaDriverEntryPointSuccess)
+            fn = reinterpret_cast<EncodeTiledFn>(p);
+        else
+            cudaGetLastError();
+    }
+    return fn;
+}
+
+// 2-D uint8 tensor [rows][row_bytes], box [box_rows][box_bytes].
+inline bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t row_bytes, uint32_t box_rows,
+                     uint32_t box_bytes, CUtensorMapSwizzle swz) {
+    EncodeTiledFn fn = encode_fn();
+    if (!fn) return false;
+    const cuuint64_t dims[2] = {row_bytes, rows};
+    const cuuint64_t strides[1] = {row_bytes};
+    const cuuint32_t box[2] = {box_bytes, box_rows};
+    const cuuint32_t estr[2] = {1, 1};
+    return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
+              CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
+              CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+inline int sm_count() {
+    static int n = 0;
+    if (!n) {
+        int dev = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
+        if (n <= 0) n = 148;
+    }
+    return n;
+}
+
+inline bool device_is_sm100() {
+    static int ok = -1;
+    if (ok < 0) {
+        int dev = 0, major = 0;
+        if (cudaGetDevice(&dev) != cudaSuccess || cudaDeviceGetAttribute(&major, cudaDevAttrComputeCapabilityMajor, dev) != cudaSuccess) {
+            cudaGetLastError();
+            return false;
+        }
+        ok = (major == 10) ? 1 : 0;
+    }
+    return ok == 1;
+}
+
+}  // namespace tc
+}  // namespace sqap
