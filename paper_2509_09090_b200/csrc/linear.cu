@@ -249,7 +249,7 @@ static size_t round256(size_t v) { return (v + 255) / 256 * 256; }
 
 namespace sqap {
 
-enum LinearPath { PATH_SIMT, PATH_TC, PATH_GEMV };
+enum LinearPath { PATH_SIMT, PATH_TC, PATH_TC_TS, PATH_GEMV };
 
 // Argument rules shared by the entry points that run a linear (everything except the activation side).
 static sqap_status check_linear_args(int M, const sqap_weights* w, const sqap_weights* w_up, const void* out,
@@ -257,7 +257,7 @@ static sqap_status check_linear_args(int M, const sqap_weights* w, const sqap_we
     if (M < 0 || !w) return SQAP_ERR_INVALID;
     if (out_dtype != SQAP_FP16 && out_dtype != SQAP_BF16 && out_dtype != SQAP_I32) return SQAP_ERR_INVALID;
     if (flags & ~allowed_flags) return SQAP_ERR_INVALID;
-    const uint32_t force = flags & (SQAP_L_FORCE_SIMT | SQAP_L_FORCE_TCGEN05 | SQAP_L_FORCE_GEMV);
+    const uint32_t force = flags & SQAP_L_FORCE_MASK;
     if ((force & (force - 1)) != 0) return SQAP_ERR_INVALID;  // at most one forced kernel
     if (w_up && (w_up->N != w->N || w_up->K != w->K || w_up->half != w->half)) return SQAP_ERR_INVALID;
     if (w_up && out_dtype == SQAP_I32) return SQAP_ERR_INVALID;
@@ -297,6 +297,9 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
     } else if (flags & SQAP_L_FORCE_TCGEN05) {
         if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
         *path = PATH_TC;
+    } else if (flags & SQAP_L_FORCE_TCGEN05_TS) {
+        if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
+        *path = PATH_TC_TS;
     } else {
         *path = a.M <= 8 ? PATH_GEMV : (tcgen05_supports(a) ? PATH_TC : PATH_SIMT);
     }
@@ -305,6 +308,7 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
 
 static sqap_status run_gemm(const LinearArgs& a, LinearPath path, cudaStream_t s) {
     if (path == PATH_TC) return launch_linear_tcgen05(a, s);
+    if (path == PATH_TC_TS) return launch_linear_tcgen05_ts(a, s);
     if (path == PATH_GEMV) {
         if (a.M == 1) launch_gemv<1>(a, s);
         else if (a.M == 2) launch_gemv<2>(a, s);
@@ -335,8 +339,7 @@ sqap_status sqap_w4a4_linear(const uint8_t* q_packed, const float* act_scales, i
                              void* workspace, size_t workspace_bytes, void* stream) {
     using namespace sqap;
     sqap_status st = check_linear_args(M, w, w_up, out, ldo, out_dtype, flags,
-                                       SQAP_L_FORCE_SIMT | SQAP_L_FORCE_TCGEN05 | SQAP_L_FORCE_GEMV |
-                                           SQAP_L_REUSE_EXPANDED);
+                                       SQAP_L_FORCE_MASK | SQAP_L_REUSE_EXPANDED);
     if (st != SQAP_OK || M == 0) return st;
     if (!q_packed || !act_scales || !workspace) return SQAP_ERR_INVALID;
     if (!aligned16(q_packed)) return SQAP_ERR_ALIGN;
@@ -369,8 +372,7 @@ sqap_status sqap_quantize_linear(const void* x, int M, int64_t ldx, const int32_
                                  int out_dtype, uint32_t lflags, void* workspace, size_t workspace_bytes,
                                  void* stream) {
     using namespace sqap;
-    sqap_status st = check_linear_args(M, w, w_up, out, ldo, out_dtype, lflags,
-                                       SQAP_L_FORCE_SIMT | SQAP_L_FORCE_TCGEN05 | SQAP_L_FORCE_GEMV);
+    sqap_status st = check_linear_args(M, w, w_up, out, ldo, out_dtype, lflags, SQAP_L_FORCE_MASK);
     if (st != SQAP_OK) return st;
     st = quantize_check_args(x, M, w->K, ldx, qflags);
     if (st != SQAP_OK || M == 0) return st;

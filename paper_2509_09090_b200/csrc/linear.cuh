@@ -39,4 +39,8 @@ __device__ __forceinline__ void store_out(void* out, int64_t idx, int out_dtype,
 sqap_status launch_linear_tcgen05(const LinearArgs& a, cudaStream_t s);
 bool tcgen05_supports(const LinearArgs& a);
 
+// tcgen05 kernel with the weight operand in tensor memory (linear_tc_ts.cu). Runs every shape the kernel
+// above runs.
+sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s);
+
 }  // namespace sqap

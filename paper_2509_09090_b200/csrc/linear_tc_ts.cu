@@ -1,0 +1,311 @@
+// tcgen05 kernel of the W4A4 linear with the weight operand in TENSOR MEMORY, for large token counts.
+//
+// D[n][m] = sum_k W[n][k] * X[m][k], weights as the 128-row MMA-M operand, tokens as the MMA-N operand
+// (BN <= 192 per tile), int8 x int8 -> int32 (kind::i8). What bounds the kernel in linear_tc.cu is shared-memory
+// bandwidth: besides the tensor core's own operand reads and the TMA writes, its unpack warps read the packed
+// weights from shared memory and write them back as int8 for the MMA to read again. Here the unpacked weights
+// never touch shared memory: the unpack warps go from the packed TMA tile through registers (two ANDs per 8
+// weights, see common.cuh) into tensor memory (tcgen05.st), and the MMA takes its A operand from there.
+// Tensor memory (512 columns): two accumulators of 192 columns (the epilogue overlaps the next tile's main
+// loop) + a ring of four 32-column weight tiles (128 int8 per lane).
+//
+// Per CTA (persistent, one per SM), warp roles:
+//   warp 0      TMA producer: per K-step of 128 codes one box of packed weights (128 rows x 64 B, 64B-swizzled)
+//               and one box of int8 activations (BN rows x 128 B, 128B-swizzled)
+//   warps 2-5   unpack: thread = one tensor-memory lane = one weight row of the tile
+//   warp 1      MMA issuer: 4 x tcgen05.mma (K = 32 each, A in tensor memory) per K-step
+//   warps 6-13  epilogue (as in linear_tc.cu)
+// Every wait on an mbarrier is bounded; on expiry the kernel records SQAP_ERR_TIMEOUT in the device status
+// word, drains and frees its tensor memory, and returns.
+#include "tc_common.cuh"
+
+namespace sqap {
+namespace tcts {
+
+using namespace tc;
+
+constexpr int BM = 128;                   // weight rows per tile (MMA M)
+constexpr int BK = 128;                   // codes of K per pipeline stage
+constexpr int BN_MAX = 192;               // tokens per tile (MMA N), runtime BN <= BN_MAX, multiple of 16
+constexpr int S = 6;                      // TMA ring: packed weights + activation tile
+constexpr int U = 4;                      // ring of unpacked weight tiles in tensor memory
+constexpr int X_BYTES = BN_MAX * BK;      // 24 KB
+constexpr int WP_BYTES = BM * BK / 2;     // 8 KB
+constexpr int OFF_X = 0;
+constexpr int OFF_WP = OFF_X + S * X_BYTES;
+constexpr int OFF_BAR = OFF_WP + S * WP_BYTES;
+constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;  // barriers + slack for 1024-byte alignment
+constexpr int TMEM_A_COL = 2 * BN_MAX;    // columns [0,192) and [192,384): accumulators; from 384: weight tiles
+constexpr int A_COLS = BK / 4;            // 32 columns hold 128 int8 per lane
+constexpr int EPI_WARPS = 8;
+constexpr int THREADS = 32 * (6 + EPI_WARPS);
+static_assert(X_BYTES % 1024 == 0 && OFF_WP % 1024 == 0, "operand tiles must be 1024-byte aligned");
+static_assert(TMEM_A_COL + U * A_COLS <= 512, "tensor memory budget");
+static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+
+// D (tensor memory) += A (tensor memory: lane = row, 4 int8 per 32-bit column) * B (shared memory descriptor).
+__device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+    asm volatile(
+        "{\n\t.reg .pred p;\n\t"
+        "setp.ne.b32 p, %4, 0;\n\t"
+        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        : "memory");
+}
+// 32 consecutive columns of this thread's tensor-memory lane.
+__device__ __forceinline__ void tc_st32(uint32_t taddr, const uint32_t* r) {
+    asm volatile(
+        "tcgen05.st.sync.aligned.32x32b.x32.b32 [%0], {%1, %2, %3, %4, %5, %6, %7, %8, %9, %10, %11, %12, %13, %14, %15, %16, "
+        "%17, %18, %19, %20, %21, %22, %23, %24, %25, %26, %27, %28, %29, %30, %31, %32};"
+        ::"r"(taddr), "r"(r[0]), "r"(r[1]), "r"(r[2]), "r"(r[3]), "r"(r[4]), "r"(r[5]), "r"(r[6]), "r"(r[7]), "r"(r[8]),
+          "r"(r[9]), "r"(r[10]), "r"(r[11]), "r"(r[12]), "r"(r[13]), "r"(r[14]), "r"(r[15]), "r"(r[16]), "r"(r[17]),
+          "r"(r[18]), "r"(r[19]), "r"(r[20]), "r"(r[21]), "r"(r[22]), "r"(r[23]), "r"(r[24]), "r"(r[25]), "r"(r[26]),
+          "r"(r[27]), "r"(r[28]), "r"(r[29]), "r"(r[30]), "r"(r[31])
+        : "memory");
+}
+__device__ __forceinline__ void tc_wait_st() { asm volatile("tcgen05.wait::st.sync.aligned;" ::: "memory"); }
+
+__global__ void __launch_bounds__(THREADS, 1)
+w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constant__ CUtensorMap tm_w_up,
+                  const __grid_constant__ CUtensorMap tm_x, Args a) {
+    extern __shared__ uint8_t smem_raw[];
+    const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
+    uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
+    const uint32_t bar0 = base + OFF_BAR;
+    auto full = [&](int s) { return bar0 + 8u * s; };                  // TMA landed (weights + activations)
+    auto x_empty = [&](int s) { return bar0 + 8u * (S + s); };         // MMAs that read the activation tile are done
+    auto wp_empty = [&](int s) { return bar0 + 8u * (2 * S + s); };    // unpack warps have read the packed weights
+    auto a_full = [&](int j) { return bar0 + 8u * (3 * S + j); };      // weight tile j is in tensor memory
+    auto a_empty = [&](int j) { return bar0 + 8u * (3 * S + U + j); };  // MMAs that read weight tile j are done
+    auto acc_full = [&](int b) { return bar0 + 8u * (3 * S + 2 * U + b); };
+    auto acc_empty = [&](int b) { return bar0 + 8u * (3 * S + 2 * U + 2 + b); };
+    constexpr int NBAR = 3 * S + 2 * U + 4;
+    volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + OFF_BAR + 8 * NBAR);
+    volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + OFF_BAR + 8 * NBAR + 8);
+
+    const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
+    const int k_steps = a.K / BK;
+    const int total_tiles = a.m_tiles * a.n_tiles;
+    const uint32_t stage_tx = static_cast<uint32_t>(WP_BYTES + a.BN * BK);
+
+    if (threadIdx.x == 0) {
+        for (int s = 0; s < S; ++s) {
+            mbar_init(full(s), 1);
+            mbar_init(x_empty(s), 1);
+            mbar_init(wp_empty(s), 4);
+        }
+        for (int j = 0; j < U; ++j) {
+            mbar_init(a_full(j), 4);
+            mbar_init(a_empty(j), 1);
+        }
+        for (int b = 0; b < 2; ++b) {
+            mbar_init(acc_full(b), 1);
+            mbar_init(acc_empty(b), EPI_WARPS);
+        }
+        abort_flag[0] = 0;
+        abort_flag[1] = 0;  // always-zero word for waits that must ignore the abort request
+        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    }
+    if (warp == 1) {
+        asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
+        asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    const uint32_t tmem_base = *tmem_slot;
+    bool failed = false;
+
+    if (warp == 0) {
+        // ---------------- TMA producer (one lane)
+        if (lane == 0) {
+            uint32_t it = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x) {
+                const int n0 = (tile % a.n_tiles) * BM, m0 = (tile / a.n_tiles) * a.BN;
+                for (int ks = 0; ks < k_steps; ++ks, ++it) {
+                    const int s = it % S;
+                    const uint32_t ph = (it / S) & 1u;
+                    if (!mbar_wait(x_empty(s), ph ^ 1u, abort_flag) || !mbar_wait(wp_empty(s), ph ^ 1u, abort_flag)) { failed = true; break; }
+                    mbar_expect_tx(full(s), stage_tx);
+                    if (a.swiglu) {
+                        tma_load_2d(base + OFF_WP + s * WP_BYTES, &tm_w, ks * (BK / 2), n0 / 2, full(s));
+                        tma_load_2d(base + OFF_WP + s * WP_BYTES + WP_BYTES / 2, &tm_w_up, ks * (BK / 2), n0 / 2, full(s));
+                    } else {
+                        tma_load_2d(base + OFF_WP + s * WP_BYTES, &tm_w, ks * (BK / 2), n0, full(s));
+                    }
+                    tma_load_2d(base + OFF_X + s * X_BYTES, &tm_x, ks * BK, m0, full(s));
+                }
+            }
+            if (failed) {
+                // drain: give every armed stage a bounded chance to land before shared memory is released
+                for (int s = 0; s < S; ++s) {
+                    const uint32_t last = it > static_cast<uint32_t>(s) ? (it - 1 - s) : 0xFFFFFFFFu;
+                    if (last != 0xFFFFFFFFu) mbar_wait(full(last % S), (last / S) & 1u, abort_flag + 1);
+                }
+            }
+        }
+    } else if (warp == 1) {
+        // ---------------- MMA issuer (one lane)
+        if (lane == 0) {
+            const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
+                                   (static_cast<uint32_t>(BM >> 4) << 24);
+            uint32_t it = 0, lt = 0;
+            for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x, ++lt) {
+                const int b = lt & 1;
+                if (!mbar_wait(acc_empty(b), ((lt >> 1) & 1u) ^ 1u, abort_flag)) { failed = true; break; }
+                tc_fence_after();
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(b * BN_MAX);
+                for (int ks = 0; ks < k_steps; ++ks, ++it) {
+                    const int s = it % S, j = it % U;
+                    // the unpack warps arrive on a_full(j) only after they saw full(s): this wait covers both operands
+                    if (!mbar_wait(a_full(j), (it / U) & 1u, abort_flag)) { failed = true; break; }
+                    tc_fence_after();
+                    const uint32_t a_tmem = tmem_base + static_cast<uint32_t>(TMEM_A_COL + j * A_COLS);
+                    const uint64_t bdesc = smem_desc_sw128(base + OFF_X + s * X_BYTES);
+#pragma unroll
+                    for (int k = 0; k < BK / 32; ++k)
+                        tc_mma_i8_ts(d_tmem, a_tmem + 8u * k, bdesc + 2u * k, idesc, (ks | k) != 0 ? 1u : 0u);
+                    tc_commit(x_empty(s));
+                    tc_commit(a_empty(j));
+                }
+                if (failed) break;
+                tc_commit(acc_full(b));
+            }
+        }
+    } else if (warp < 6) {
+        // ---------------- unpack warps: thread = one tensor-memory lane = one weight row of the tile
+        const int quad = warp & 3;                 // the lane quadrant this warp may write
+        const int L = quad * 32 + lane;            // tensor-memory lane
+        // Source row of the packed stage. Plain: row L. SwiGLU: the stage holds 64 gate rows then 64 up rows;
+        // within each quadrant lanes 0-15 take gate rows and lanes 16-31 the up rows of the same 16 channels.
+        const int src_row = a.swiglu ? (quad * 16 + (lane & 15) + ((lane >> 4) << 6)) : L;
+        // 64-byte rows under the 64B TMA swizzle: 16-byte chunk c of row r sits at chunk c ^ ((r >> 1) & 3).
+        // Consecutive rows then hit different banks for the same c, so the register a chunk lands in is fixed.
+        const int sw = (src_row >> 1) & 3;
+        uint32_t it = 0;
+        for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x) {
+            for (int ks = 0; ks < k_steps; ++ks, ++it) {
+                const int s = it % S, j = it % U;
+                const bool ok = mbar_wait(full(s), (it / S) & 1u, abort_flag) &&
+                                mbar_wait(a_empty(j), ((it / U) & 1u) ^ 1u, abort_flag);
+                if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                tc_fence_after();
+                const uint8_t* src = sm + OFF_WP + s * WP_BYTES + src_row * 64;
+                uint32_t r[32];   // column q holds codes k = 4q .. 4q+3 of the row
+#pragma unroll
+                for (int c = 0; c < 4; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(src + ((c ^ sw) << 4));
+                    r[4 * c + 0] = v.x & 0x0F0F0F0Fu; r[4 * c + 1] = v.y & 0x0F0F0F0Fu;      // codes 16c .. 16c+15 (+8)
+                    r[4 * c + 2] = v.z & 0x0F0F0F0Fu; r[4 * c + 3] = v.w & 0x0F0F0F0Fu;
+                    r[16 + 4 * c + 0] = v.x & 0xF0F0F0F0u; r[16 + 4 * c + 1] = v.y & 0xF0F0F0F0u;  // codes 64+16c .. (x16)
+                    r[16 + 4 * c + 2] = v.z & 0xF0F0F0F0u; r[16 + 4 * c + 3] = v.w & 0xF0F0F0F0u;
+                }
+                tc_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(TMEM_A_COL + j * A_COLS), r);
+                tc_wait_st();
+                tc_fence_before();
+                __syncwarp();
+                if (lane == 0) {
+                    mbar_arrive(wp_empty(s));
+                    mbar_arrive(a_full(j));
+                }
+            }
+        }
+    } else {
+        // ---------------- epilogue warps: warp % 4 selects the 32-lane quadrant of tensor memory
+        const int quad = warp & 3;
+        const int row = quad * 32 + lane;
+        const int split = ((a.BN / 16 + 1) / 2) * 16;  // first token of the second half of the tile
+        const int c_begin = (warp - 6) < 4 ? 0 : split;
+        const int c_end = (warp - 6) < 4 ? split : a.BN;
+        uint32_t lt = 0;
+        for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x, ++lt) {
+            const int b = lt & 1;
+            const int n0 = (tile % a.n_tiles) * BM, m0 = (tile / a.n_tiles) * a.BN;
+            if (!__all_sync(0xffffffffu, mbar_wait(acc_full(b), (lt >> 1) & 1u, abort_flag))) { failed = true; break; }
+            tc_fence_after();
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(b * BN_MAX);
+            int n;
+            float sw;
+            bool n_ok;
+            if (a.swiglu) {
+                n = n0 / 2 + quad * 16 + (lane & 15);      // lanes 0-15 of a quadrant: gate, 16-31: up, same channels
+                n_ok = n < a.N;
+                sw = n_ok ? __half2float((lane & 16) ? a.w_up_scales[n] : a.w_scales[n]) : 0.0f;
+            } else {
+                n = n0 + row;
+                n_ok = n < a.N;
+                sw = n_ok ? __half2float(a.w_scales[n]) : 0.0f;
+            }
+            if (a.swiglu) {
+                if (a.out_dtype == SQAP_FP16) epilogue_tile<SQAP_FP16, true, 16>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
+                else epilogue_tile<SQAP_BF16, true, 16>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
+            } else {
+                if (a.out_dtype == SQAP_FP16) epilogue_tile<SQAP_FP16, false>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
+                else if (a.out_dtype == SQAP_BF16) epilogue_tile<SQAP_BF16, false>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
+                else epilogue_tile<SQAP_I32, false>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
+            }
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) mbar_arrive(acc_empty(b));
+        }
+    }
+
+    if (failed) {
+        *abort_flag = 1;
+        atomicOr(a.status, SQAP_ERR_TIMEOUT);
+    }
+    tc_fence_before();
+    __syncthreads();
+    tc_fence_after();
+    if (warp == 1) {
+        asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
+    }
+}
+
+}  // namespace tcts
+
+sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s) {
+    using namespace tcts;
+    Args k;
+    k.bias_sum = a.bias_sum;
+    k.act_scales = a.act_scales;
+    k.w_scales = a.w_scales;
+    k.w_up_scales = a.w_up_scales;
+    k.out = a.out;
+    k.ldo = a.ldo;
+    k.M = a.M;
+    k.N = a.N;
+    k.K = a.K;
+    k.m_tiles = (a.M + BN_MAX - 1) / BN_MAX;
+    const int per = (a.M + k.m_tiles - 1) / k.m_tiles;
+    k.BN = (per + 15) / 16 * 16;
+    k.swiglu = a.w_up ? 1 : 0;
+    k.n_tiles = k.swiglu ? (2 * a.N + BM - 1) / BM : (a.N + BM - 1) / BM;
+    k.out_dtype = a.out_dtype;
+    k.status = device_status_word();
+    if (!k.status) return SQAP_ERR_CUDA;
+
+    CUtensorMap tm_w, tm_u, tm_x;
+    const uint32_t w_box_rows = k.swiglu ? BM / 2 : BM;
+    if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BK / 2, CU_TENSOR_MAP_SWIZZLE_64B)) return SQAP_ERR_CUDA;
+    if (!make_map(&tm_u, k.swiglu ? a.w_up : a.w, a.N, a.K / 2, w_box_rows, BK / 2, CU_TENSOR_MAP_SWIZZLE_64B))
+        return SQAP_ERR_CUDA;
+    if (!make_map(&tm_x, a.x8, a.M, a.K, k.BN, BK, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
+
+    static bool attr_set = false;
+    if (!attr_set) {
+        cudaError_t e = cudaFuncSetAttribute(w4a4_tc_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
+        if (e != cudaSuccess) {
+            note_cuda_error(e);
+            return SQAP_ERR_CUDA;
+        }
+        attr_set = true;
+    }
+    const int tiles = k.m_tiles * k.n_tiles;
+    const int grid = tiles < sm_count() ? tiles : sm_count();
+    w4a4_tc_ts_kernel<<<grid, THREADS, SMEM_BYTES, s>>>(tm_w, tm_u, tm_x, k);
+    count_launch();
+    return check_launch();
+}
+
+}  // namespace sqap

@@ -103,12 +103,12 @@ __device__ __forceinline__ float silu_mul_fast(float g, float u) { return __fdiv
 // with SwiGLU the even lane of a pair holds the gate and the odd lane the up projection of channel n) and
 // walks the tokens [c_begin, c_end) of the tile 16 at a time; the per-token bias sums and scales of a chunk
 // are fetched by lanes 0-15 with one coalesced load each (one chunk ahead) and broadcast by shuffle.
-template <int OUT, bool SWIGLU>
+template <int OUT, bool SWIGLU, int XCHG = 1>
 __device__ __forceinline__ void epilogue_tile(const Args& a, uint32_t taddr, int m0, int c_begin, int c_end, int n,
                                               bool n_ok, float sw, int lane) {
     constexpr int ESZ = OUT == SQAP_I32 ? 4 : 2;
     const int ml = lane & 15;
-    const bool odd = (lane & 1) != 0;
+    const bool odd = (lane & XCHG) != 0;   // SwiGLU: this lane holds the up projection, its partner (lane ^ XCHG) the gate
     const int64_t row_bytes = a.ldo * ESZ;
     int mm = m0 + c_begin + ml;
     int bs_next = mm < a.M ? (__ldg(a.bias_sum + mm) << 7) : 0;
@@ -135,7 +135,7 @@ __device__ __forceinline__ void epilogue_tile(const Args& a, uint32_t taddr, int
                                                      __shfl_sync(0xffffffffu, sx_cur, j)), sw);
                 const float y1 = __fmul_rn(__fmul_rn(static_cast<float>((static_cast<int>(v[j + 1]) - __shfl_sync(0xffffffffu, bs_cur, j + 1)) >> 4),
                                                      __shfl_sync(0xffffffffu, sx_cur, j + 1)), sw);
-                const float got = __shfl_xor_sync(0xffffffffu, odd ? y0 : y1, 1);
+                const float got = __shfl_xor_sync(0xffffffffu, odd ? y0 : y1, XCHG);
                 const float h = odd ? silu_mul_fast(got, y1) : silu_mul_fast(y0, got);
                 const int jj = odd ? j + 1 : j;
                 if (n_ok && jj < valid) {
