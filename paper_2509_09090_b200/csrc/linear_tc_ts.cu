@@ -7,13 +7,16 @@
 // never touch shared memory: the unpack warps go from the packed TMA tile through registers (two ANDs per 8
 // weights, see common.cuh) into tensor memory (tcgen05.st), and the MMA takes its A operand from there.
 // Tensor memory (512 columns): two accumulators of 192 columns (the epilogue overlaps the next tile's main
-// loop) + a ring of four 32-column weight tiles (128 int8 per lane).
+// loop) + a ring of two 64-column weight tiles (256 int8 per lane).
+// One thread issues every MMA, and a tcgen05.mma, a tcgen05.commit or an mbarrier wait each cost it some 60
+// cycles: a pipeline stage therefore covers 256 codes of K (8 MMAs of 96 cycles) per wait and per commit, and
+// a single barrier per stage ("done") releases both the shared-memory slot and the tensor-memory weight tile.
 //
 // Per CTA (persistent, one per SM), warp roles:
-//   warp 0      TMA producer: per K-step of 128 codes one box of packed weights (128 rows x 64 B, 64B-swizzled)
-//               and one box of int8 activations (BN rows x 128 B, 128B-swizzled)
+//   warp 0      TMA producer: per stage two boxes of packed weights (128 rows x 64 B, 64B-swizzled) and two
+//               boxes of int8 activations (BN rows x 128 B, 128B-swizzled)
 //   warps 2-5   unpack: thread = one tensor-memory lane = one weight row of the tile
-//   warp 1      MMA issuer: 4 x tcgen05.mma (K = 32 each, A in tensor memory) per K-step
+//   warp 1      MMA issuer: 8 x tcgen05.mma (K = 32 each, A in tensor memory) per stage
 //   warps 6-13  epilogue (as in linear_tc.cu)
 // Every wait on an mbarrier is bounded; on expiry the kernel records SQAP_ERR_TIMEOUT in the device status
 // word, drains and frees its tensor memory, and returns.
@@ -25,23 +28,25 @@ namespace tcts {
 using namespace tc;
 
 constexpr int BM = 128;                   // weight rows per tile (MMA M)
-constexpr int BK = 128;                   // codes of K per pipeline stage
+constexpr int BKH = 128;                  // codes of K per TMA box / per block of the packed weight layout
+constexpr int BK = 2 * BKH;               // codes of K per pipeline stage
 constexpr int BN_MAX = 192;               // tokens per tile (MMA N), runtime BN <= BN_MAX, multiple of 16
-constexpr int S = 6;                      // TMA ring: packed weights + activation tile
-constexpr int U = 4;                      // ring of unpacked weight tiles in tensor memory
-constexpr int X_BYTES = BN_MAX * BK;      // 24 KB
-constexpr int WP_BYTES = BM * BK / 2;     // 8 KB
+constexpr int S = 3;                      // TMA ring: packed weights + activation tile
+constexpr int U = 2;                      // ring of unpacked weight tiles in tensor memory
+constexpr int XH_BYTES = BN_MAX * BKH;    // 24 KB: one 128-code half of a stage's activation tile
+constexpr int WPH_BYTES = BM * BKH / 2;   // 8 KB: one half of a stage's packed weights
 constexpr int OFF_X = 0;
-constexpr int OFF_WP = OFF_X + S * X_BYTES;
-constexpr int OFF_BAR = OFF_WP + S * WP_BYTES;
+constexpr int OFF_WP = OFF_X + S * 2 * XH_BYTES;
+constexpr int OFF_BAR = OFF_WP + S * 2 * WPH_BYTES;
 constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;  // barriers + slack for 1024-byte alignment
 constexpr int TMEM_A_COL = 2 * BN_MAX;    // columns [0,192) and [192,384): accumulators; from 384: weight tiles
-constexpr int A_COLS = BK / 4;            // 32 columns hold 128 int8 per lane
+constexpr int A_COLS = BK / 4;            // 64 columns hold 256 int8 per lane
 constexpr int EPI_WARPS = 8;
 constexpr int THREADS = 32 * (6 + EPI_WARPS);
-static_assert(X_BYTES % 1024 == 0 && OFF_WP % 1024 == 0, "operand tiles must be 1024-byte aligned");
+static_assert(XH_BYTES % 1024 == 0 && OFF_WP % 1024 == 0, "operand tiles must be 1024-byte aligned");
 static_assert(TMEM_A_COL + U * A_COLS <= 512, "tensor memory budget");
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
+static_assert(S > U, "a stage's done barrier must not wrap before the unpack warps have seen it");
 
 // D (tensor memory) += A (tensor memory: lane = row, 4 int8 per 32-bit column) * B (shared memory descriptor).
 __device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
@@ -73,30 +78,28 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t bar0 = base + OFF_BAR;
     auto full = [&](int s) { return bar0 + 8u * s; };                  // TMA landed (weights + activations)
-    auto x_empty = [&](int s) { return bar0 + 8u * (S + s); };         // MMAs that read the activation tile are done
+    auto done = [&](int s) { return bar0 + 8u * (S + s); };            // the MMAs of the stage in slot s are done
     auto wp_empty = [&](int s) { return bar0 + 8u * (2 * S + s); };    // unpack warps have read the packed weights
     auto a_full = [&](int j) { return bar0 + 8u * (3 * S + j); };      // weight tile j is in tensor memory
-    auto a_empty = [&](int j) { return bar0 + 8u * (3 * S + U + j); };  // MMAs that read weight tile j are done
-    auto acc_full = [&](int b) { return bar0 + 8u * (3 * S + 2 * U + b); };
-    auto acc_empty = [&](int b) { return bar0 + 8u * (3 * S + 2 * U + 2 + b); };
-    constexpr int NBAR = 3 * S + 2 * U + 4;
+    auto acc_full = [&](int b) { return bar0 + 8u * (3 * S + U + b); };
+    auto acc_empty = [&](int b) { return bar0 + 8u * (3 * S + U + 2 + b); };
+    constexpr int NBAR = 3 * S + U + 4;
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + OFF_BAR + 8 * NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + OFF_BAR + 8 * NBAR + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
-    const int k_steps = a.K / BK;
+    const int k_steps = (a.K + BK - 1) / BK;   // a last half-stage past K is zero-filled by TMA and adds nothing
     const int total_tiles = a.m_tiles * a.n_tiles;
-    const uint32_t stage_tx = static_cast<uint32_t>(WP_BYTES + a.BN * BK);
+    const uint32_t stage_tx = static_cast<uint32_t>(2 * (WPH_BYTES + a.BN * BKH));
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
             mbar_init(full(s), 1);
-            mbar_init(x_empty(s), 1);
+            mbar_init(done(s), 1);
             mbar_init(wp_empty(s), 4);
         }
         for (int j = 0; j < U; ++j) {
             mbar_init(a_full(j), 4);
-            mbar_init(a_empty(j), 1);
         }
         for (int b = 0; b < 2; ++b) {
             mbar_init(acc_full(b), 1);
@@ -125,15 +128,20 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
                 for (int ks = 0; ks < k_steps; ++ks, ++it) {
                     const int s = it % S;
                     const uint32_t ph = (it / S) & 1u;
-                    if (!mbar_wait(x_empty(s), ph ^ 1u, abort_flag) || !mbar_wait(wp_empty(s), ph ^ 1u, abort_flag)) { failed = true; break; }
+                    if (!mbar_wait(done(s), ph ^ 1u, abort_flag) || !mbar_wait(wp_empty(s), ph ^ 1u, abort_flag)) { failed = true; break; }
                     mbar_expect_tx(full(s), stage_tx);
-                    if (a.swiglu) {
-                        tma_load_2d(base + OFF_WP + s * WP_BYTES, &tm_w, ks * (BK / 2), n0 / 2, full(s));
-                        tma_load_2d(base + OFF_WP + s * WP_BYTES + WP_BYTES / 2, &tm_w_up, ks * (BK / 2), n0 / 2, full(s));
-                    } else {
-                        tma_load_2d(base + OFF_WP + s * WP_BYTES, &tm_w, ks * (BK / 2), n0, full(s));
+#pragma unroll
+                    for (int h = 0; h < 2; ++h) {
+                        const uint32_t wp = base + OFF_WP + (2 * s + h) * WPH_BYTES;
+                        const int kc = ks * BK + h * BKH;   // first code of this half
+                        if (a.swiglu) {
+                            tma_load_2d(wp, &tm_w, kc / 2, n0 / 2, full(s));
+                            tma_load_2d(wp + WPH_BYTES / 2, &tm_w_up, kc / 2, n0 / 2, full(s));
+                        } else {
+                            tma_load_2d(wp, &tm_w, kc / 2, n0, full(s));
+                        }
+                        tma_load_2d(base + OFF_X + (2 * s + h) * XH_BYTES, &tm_x, kc, m0, full(s));
                     }
-                    tma_load_2d(base + OFF_X + s * X_BYTES, &tm_x, ks * BK, m0, full(s));
                 }
             }
             if (failed) {
@@ -161,12 +169,14 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
                     if (!mbar_wait(a_full(j), (it / U) & 1u, abort_flag)) { failed = true; break; }
                     tc_fence_after();
                     const uint32_t a_tmem = tmem_base + static_cast<uint32_t>(TMEM_A_COL + j * A_COLS);
-                    const uint64_t bdesc = smem_desc_sw128(base + OFF_X + s * X_BYTES);
 #pragma unroll
-                    for (int k = 0; k < BK / 32; ++k)
-                        tc_mma_i8_ts(d_tmem, a_tmem + 8u * k, bdesc + 2u * k, idesc, (ks | k) != 0 ? 1u : 0u);
-                    tc_commit(x_empty(s));
-                    tc_commit(a_empty(j));
+                    for (int h = 0; h < 2; ++h) {
+                        const uint64_t bdesc = smem_desc_sw128(base + OFF_X + (2 * s + h) * XH_BYTES);
+#pragma unroll
+                        for (int k = 0; k < BKH / 32; ++k)
+                            tc_mma_i8_ts(d_tmem, a_tmem + 32u * h + 8u * k, bdesc + 2u * k, idesc, (ks | h | k) != 0 ? 1u : 0u);
+                    }
+                    tc_commit(done(s));
                 }
                 if (failed) break;
                 tc_commit(acc_full(b));
@@ -186,21 +196,26 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
         for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x) {
             for (int ks = 0; ks < k_steps; ++ks, ++it) {
                 const int s = it % S, j = it % U;
-                const bool ok = mbar_wait(full(s), (it / S) & 1u, abort_flag) &&
-                                mbar_wait(a_empty(j), ((it / U) & 1u) ^ 1u, abort_flag);
+                // weight tile j was last read by the MMAs of stage it - U, whose completion is done((it - U) % S)
+                bool ok = mbar_wait(full(s), (it / S) & 1u, abort_flag);
+                if (ok && it >= U) ok = mbar_wait(done((it - U) % S), ((it - U) / S) & 1u, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 tc_fence_after();
-                const uint8_t* src = sm + OFF_WP + s * WP_BYTES + src_row * 64;
-                uint32_t r[32];   // column q holds codes k = 4q .. 4q+3 of the row
 #pragma unroll
-                for (int c = 0; c < 4; ++c) {
-                    const uint4 v = *reinterpret_cast<const uint4*>(src + ((c ^ sw) << 4));
-                    r[4 * c + 0] = v.x & 0x0F0F0F0Fu; r[4 * c + 1] = v.y & 0x0F0F0F0Fu;      // codes 16c .. 16c+15 (+8)
-                    r[4 * c + 2] = v.z & 0x0F0F0F0Fu; r[4 * c + 3] = v.w & 0x0F0F0F0Fu;
-                    r[16 + 4 * c + 0] = v.x & 0xF0F0F0F0u; r[16 + 4 * c + 1] = v.y & 0xF0F0F0F0u;  // codes 64+16c .. (x16)
-                    r[16 + 4 * c + 2] = v.z & 0xF0F0F0F0u; r[16 + 4 * c + 3] = v.w & 0xF0F0F0F0u;
+                for (int h = 0; h < 2; ++h) {
+                    const uint8_t* src = sm + OFF_WP + (2 * s + h) * WPH_BYTES + src_row * 64;
+                    uint32_t r[32];   // column q holds codes k = 4q .. 4q+3 of this half of the row
+#pragma unroll
+                    for (int c = 0; c < 4; ++c) {
+                        const uint4 v = *reinterpret_cast<const uint4*>(src + ((c ^ sw) << 4));
+                        r[4 * c + 0] = v.x & 0x0F0F0F0Fu; r[4 * c + 1] = v.y & 0x0F0F0F0Fu;      // codes 16c .. 16c+15 (+8)
+                        r[4 * c + 2] = v.z & 0x0F0F0F0Fu; r[4 * c + 3] = v.w & 0x0F0F0F0Fu;
+                        r[16 + 4 * c + 0] = v.x & 0xF0F0F0F0u; r[16 + 4 * c + 1] = v.y & 0xF0F0F0F0u;  // codes 64+16c .. (x16)
+                        r[16 + 4 * c + 2] = v.z & 0xF0F0F0F0u; r[16 + 4 * c + 3] = v.w & 0xF0F0F0F0u;
+                    }
+                    tc_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
+                                static_cast<uint32_t>(TMEM_A_COL + j * A_COLS + 32 * h), r);
                 }
-                tc_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(TMEM_A_COL + j * A_COLS), r);
                 tc_wait_st();
                 tc_fence_before();
                 __syncwarp();
@@ -287,10 +302,10 @@ sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s) {
 
     CUtensorMap tm_w, tm_u, tm_x;
     const uint32_t w_box_rows = k.swiglu ? BM / 2 : BM;
-    if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BK / 2, CU_TENSOR_MAP_SWIZZLE_64B)) return SQAP_ERR_CUDA;
-    if (!make_map(&tm_u, k.swiglu ? a.w_up : a.w, a.N, a.K / 2, w_box_rows, BK / 2, CU_TENSOR_MAP_SWIZZLE_64B))
+    if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B)) return SQAP_ERR_CUDA;
+    if (!make_map(&tm_u, k.swiglu ? a.w_up : a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B))
         return SQAP_ERR_CUDA;
-    if (!make_map(&tm_x, a.x8, a.M, a.K, k.BN, BK, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
+    if (!make_map(&tm_x, a.x8, a.M, a.K, k.BN, BKH, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
 
     static bool attr_set = false;
     if (!attr_set) {
