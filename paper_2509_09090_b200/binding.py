@@ -17,7 +17,7 @@ SQAP_STATIC_WORKSPACE_BYTES = 4 * 1024 * 1024 + 8192
 SQAP_FP16, SQAP_BF16, SQAP_I32 = 0, 1, 2
 SQAP_Q_ROTATE = 1
 SQAP_W_ROTATED = 1
-SQAP_L_FORCE_SIMT, SQAP_L_FORCE_TCGEN05, SQAP_L_FORCE_GEMV, SQAP_L_REUSE_EXPANDED, SQAP_L_FORCE_TCGEN05_TS = 1, 2, 4, 8, 16
+SQAP_L_FORCE_SIMT, SQAP_L_FORCE_TCGEN05, SQAP_L_FORCE_GEMV, SQAP_L_REUSE_EXPANDED, SQAP_L_FORCE_TCGEN05_TS, SQAP_L_FORCE_TCGEN05_PAIR = 1, 2, 4, 8, 16, 32
 
 EXPORTS = ("sqap_pack_weights", "sqap_free_weights", "sqap_weights_info", "sqap_unpack_weights",
            "sqap_quantize_act", "sqap_workspace_bytes", "sqap_w4a4_linear", "sqap_w4a4_linear_static",

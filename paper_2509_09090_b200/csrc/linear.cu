@@ -249,7 +249,7 @@ static size_t round256(size_t v) { return (v + 255) / 256 * 256; }
 
 namespace sqap {
 
-enum LinearPath { PATH_SIMT, PATH_TC, PATH_TC_TS, PATH_GEMV };
+enum LinearPath { PATH_SIMT, PATH_TC, PATH_TC_TS, PATH_TC_PAIR, PATH_GEMV };
 
 // Argument rules shared by the entry points that run a linear (everything except the activation side).
 static sqap_status check_linear_args(int M, const sqap_weights* w, const sqap_weights* w_up, const void* out,
@@ -300,6 +300,9 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
     } else if (flags & SQAP_L_FORCE_TCGEN05_TS) {
         if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
         *path = PATH_TC_TS;
+    } else if (flags & SQAP_L_FORCE_TCGEN05_PAIR) {
+        if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
+        *path = PATH_TC_PAIR;
     } else {
         *path = a.M <= 8 ? PATH_GEMV : (tcgen05_supports(a) ? PATH_TC : PATH_SIMT);
     }
@@ -309,6 +312,7 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
 static sqap_status run_gemm(const LinearArgs& a, LinearPath path, cudaStream_t s) {
     if (path == PATH_TC) return launch_linear_tcgen05(a, s);
     if (path == PATH_TC_TS) return launch_linear_tcgen05_ts(a, s);
+    if (path == PATH_TC_PAIR) return launch_linear_tcgen05_pair(a, s);
     if (path == PATH_GEMV) {
         if (a.M == 1) launch_gemv<1>(a, s);
         else if (a.M == 2) launch_gemv<2>(a, s);

@@ -43,4 +43,7 @@ bool tcgen05_supports(const LinearArgs& a);
 // above runs.
 sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s);
 
+// The same on CTA pairs (linear_tc_pair.cu): the large-M kernel. Runs every shape the kernels above run.
+sqap_status launch_linear_tcgen05_pair(const LinearArgs& a, cudaStream_t s);
+
 }  // namespace sqap

@@ -190,8 +190,8 @@ def test_linear_tcgen05_forced(M, N, K, swiglu):
     x = wl.activations(25, M + K, M, K, max(1, K // 100), 20.0)
     g = (wl.weight_codes(25, N + K, N, K), wl.weight_scales(25, N + K, N, mult=0.5))
     u = (wl.weight_codes(25, N + K + 1, N, K), wl.weight_scales(25, N + K + 1, N, mult=0.5)) if swiglu else None
-    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS])
-    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS], bf16=True)
+    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS, B.SQAP_L_FORCE_TCGEN05_PAIR])
+    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS, B.SQAP_L_FORCE_TCGEN05_PAIR], bf16=True)
 
 
 @pytest.mark.parametrize("M,N,K,swiglu", [(1300, 3500, 384, False), (1000, 2368, 256, True)])
@@ -201,7 +201,7 @@ def test_linear_tcgen05_many_tiles(M, N, K, swiglu):
     x = wl.activations(26, M + K, M, K, max(1, K // 100), 20.0)
     g = (wl.weight_codes(26, N + K, N, K), wl.weight_scales(26, N + K, N, mult=0.5))
     u = (wl.weight_codes(26, N + K + 1, N, K), wl.weight_scales(26, N + K + 1, N, mult=0.5)) if swiglu else None
-    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS])
+    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS, B.SQAP_L_FORCE_TCGEN05_PAIR])
 
 
 @pytest.mark.parametrize("K", [64, 128, 256, 512, 4096])
