@@ -50,12 +50,15 @@ static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 static_assert(S > U, "a stage's done barrier must not wrap before the unpack warps have seen it");
 
 // D (tensor memory) += A (tensor memory: lane = row, 4 int8 per 32-bit column) * B (shared memory descriptor).
-__device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// Issued by the lane(s) with issue != 0 of a converged warp.
+__device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate,
+                                             uint32_t issue) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::2.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(issue)
         : "memory");
 }
 // 32 consecutive columns of this thread's tensor-memory lane.
@@ -100,10 +103,12 @@ __device__ __forceinline__ void tma_load_2d_pair(uint32_t dst, const CUtensorMap
         : "memory");
 }
 // Arrives (once) on the barrier at this offset in both CTAs of the pair when all MMAs issued so far are done.
-__device__ __forceinline__ void tc_commit_pair(uint32_t bar) {
+__device__ __forceinline__ void tc_commit_pair(uint32_t bar, uint32_t issue) {
     asm volatile(
-        "tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;"
-        ::"r"(bar), "h"(static_cast<uint16_t>(3))
+        "{\n\t.reg .pred q;\n\t"
+        "setp.ne.b32 q, %2, 0;\n\t"
+        "@q tcgen05.commit.cta_group::2.mbarrier::arrive::one.shared::cluster.multicast::cluster.b64 [%0], %1;\n\t}"
+        ::"r"(bar), "h"(static_cast<uint16_t>(3)), "r"(issue)
         : "memory");
 }
 
@@ -202,20 +207,21 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer (one lane)
-        if (lane == 0 && rank == 0) {
+        // ---------------- MMA issuer (leader CTA): the whole warp walks the loop, one elected lane issues
+        if (rank == 0) {
+            const uint32_t issue = elect_one();
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
                                    (static_cast<uint32_t>((2 * BM) >> 4) << 24);
             uint32_t it = 0, lt = 0;
             for (int tile = pair; tile < total_tiles && !failed; tile += n_pairs, ++lt) {
                 const int b = lt & 1;
-                if (!mbar_wait(acc_empty(b), ((lt >> 1) & 1u) ^ 1u, abort_flag)) { failed = true; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(acc_empty(b), ((lt >> 1) & 1u) ^ 1u, abort_flag))) { failed = true; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(b * BN_MAX);
                 for (int ks = 0; ks < k_steps; ++ks, ++it) {
                     const int s = it % S, j = it % U;
-                    if (!mbar_wait(x_full(s), (it / S) & 1u, abort_flag) ||
-                        !mbar_wait(a_full(j), (it / U) & 1u, abort_flag)) { failed = true; break; }
+                    const bool ok = mbar_wait(x_full(s), (it / S) & 1u, abort_flag) && mbar_wait(a_full(j), (it / U) & 1u, abort_flag);
+                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                     tc_fence_after();
                     const uint32_t a_tmem = tmem_base + static_cast<uint32_t>(TMEM_A_COL + j * A_COLS);
 #pragma unroll
@@ -223,12 +229,12 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
                         const uint64_t bdesc = smem_desc_sw128(base + OFF_X + (2 * s + h) * XH_BYTES);
 #pragma unroll
                         for (int k = 0; k < BKH / 32; ++k)
-                            tc_mma_i8_ts(d_tmem, a_tmem + 32u * h + 8u * k, bdesc + 2u * k, idesc, (ks | h | k) != 0 ? 1u : 0u);
+                            tc_mma_i8_ts(d_tmem, a_tmem + 32u * h + 8u * k, bdesc + 2u * k, idesc, (ks | h | k) != 0 ? 1u : 0u, issue);
                     }
-                    tc_commit_pair(done(s));
+                    tc_commit_pair(done(s), issue);
                 }
                 if (failed) break;
-                tc_commit_pair(acc_full(b));
+                tc_commit_pair(acc_full(b), issue);
             }
         }
     } else if (warp < 6) {

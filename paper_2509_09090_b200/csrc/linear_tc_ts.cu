@@ -49,12 +49,15 @@ static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 static_assert(S > U, "a stage's done barrier must not wrap before the unpack warps have seen it");
 
 // D (tensor memory) += A (tensor memory: lane = row, 4 int8 per 32-bit column) * B (shared memory descriptor).
-__device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate) {
+// Issued by the lane(s) with issue != 0 of a converged warp.
+__device__ __forceinline__ void tc_mma_i8_ts(uint32_t d_tmem, uint32_t a_tmem, uint64_t bdesc, uint32_t idesc, uint32_t accumulate,
+                                             uint32_t issue) {
     asm volatile(
-        "{\n\t.reg .pred p;\n\t"
+        "{\n\t.reg .pred p, q;\n\t"
         "setp.ne.b32 p, %4, 0;\n\t"
-        "tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
-        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate)
+        "setp.ne.b32 q, %5, 0;\n\t"
+        "@q tcgen05.mma.cta_group::1.kind::i8 [%0], [%1], %2, %3, p;\n\t}"
+        ::"r"(d_tmem), "r"(a_tmem), "l"(bdesc), "r"(idesc), "r"(accumulate), "r"(issue)
         : "memory");
 }
 // 32 consecutive columns of this thread's tensor-memory lane.
@@ -153,20 +156,21 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
             }
         }
     } else if (warp == 1) {
-        // ---------------- MMA issuer (one lane)
-        if (lane == 0) {
+        // ---------------- MMA issuer: the whole warp walks the loop, one elected lane issues
+        {
+            const uint32_t issue = elect_one();
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
                                    (static_cast<uint32_t>(BM >> 4) << 24);
             uint32_t it = 0, lt = 0;
             for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x, ++lt) {
                 const int b = lt & 1;
-                if (!mbar_wait(acc_empty(b), ((lt >> 1) & 1u) ^ 1u, abort_flag)) { failed = true; break; }
+                if (!__all_sync(0xffffffffu, mbar_wait(acc_empty(b), ((lt >> 1) & 1u) ^ 1u, abort_flag))) { failed = true; break; }
                 tc_fence_after();
                 const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(b * BN_MAX);
                 for (int ks = 0; ks < k_steps; ++ks, ++it) {
                     const int s = it % S, j = it % U;
                     // the unpack warps arrive on a_full(j) only after they saw full(s): this wait covers both operands
-                    if (!mbar_wait(a_full(j), (it / U) & 1u, abort_flag)) { failed = true; break; }
+                    if (!__all_sync(0xffffffffu, mbar_wait(a_full(j), (it / U) & 1u, abort_flag))) { failed = true; break; }
                     tc_fence_after();
                     const uint32_t a_tmem = tmem_base + static_cast<uint32_t>(TMEM_A_COL + j * A_COLS);
 #pragma unroll
@@ -174,12 +178,12 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
                         const uint64_t bdesc = smem_desc_sw128(base + OFF_X + (2 * s + h) * XH_BYTES);
 #pragma unroll
                         for (int k = 0; k < BKH / 32; ++k)
-                            tc_mma_i8_ts(d_tmem, a_tmem + 32u * h + 8u * k, bdesc + 2u * k, idesc, (ks | h | k) != 0 ? 1u : 0u);
+                            tc_mma_i8_ts(d_tmem, a_tmem + 32u * h + 8u * k, bdesc + 2u * k, idesc, (ks | h | k) != 0 ? 1u : 0u, issue);
                     }
-                    tc_commit(done(s));
+                    tc_commit_if(done(s), issue);
                 }
                 if (failed) break;
-                tc_commit(acc_full(b));
+                tc_commit_if(acc_full(b), issue);
             }
         }
     } else if (warp < 6) {
