@@ -304,7 +304,7 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
         if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
         *path = PATH_TC_PAIR;
     } else {
-        *path = a.M <= 8 ? PATH_GEMV : (tcgen05_supports(a) ? PATH_TC : PATH_SIMT);
+        *path = a.M <= 8 ? PATH_GEMV : (tcgen05_supports(a) ? (a.M >= 512 ? PATH_TC_PAIR : PATH_TC) : PATH_SIMT);
     }
     return SQAP_OK;
 }

@@ -347,21 +347,11 @@ sqap_status launch_linear_tcgen05_pair(const LinearArgs& a, cudaStream_t s) {
     k.M = a.M;
     k.N = a.N;
     k.K = a.K;
-    k.m_tiles = (a.M + BN_MAX - 1) / BN_MAX;
-    const int per = (a.M + k.m_tiles - 1) / k.m_tiles;
-    k.BN = (per + 15) / 16 * 16;
     k.swiglu = a.w_up ? 1 : 0;
     k.n_tiles = k.swiglu ? (2 * a.N + 2 * BM - 1) / (2 * BM) : (a.N + 2 * BM - 1) / (2 * BM);
     k.out_dtype = a.out_dtype;
     k.status = device_status_word();
     if (!k.status) return SQAP_ERR_CUDA;
-
-    CUtensorMap tm_w, tm_u, tm_x;
-    const uint32_t w_box_rows = k.swiglu ? BM / 2 : BM;
-    if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B)) return SQAP_ERR_CUDA;
-    if (!make_map(&tm_u, k.swiglu ? a.w_up : a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B))
-        return SQAP_ERR_CUDA;
-    if (!make_map(&tm_x, a.x8, a.M, a.K, k.BN / 2, BKH, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
 
     static bool attr_set = false;
     if (!attr_set) {
@@ -394,6 +384,14 @@ sqap_status launch_linear_tcgen05_pair(const LinearArgs& a, cudaStream_t s) {
         }
         max_pairs = n;
     }
+    choose_token_tiles(a.M, k.n_tiles, max_pairs, BN_MAX, &k.m_tiles, &k.BN);
+    CUtensorMap tm_w, tm_u, tm_x;
+    const uint32_t w_box_rows = k.swiglu ? BM / 2 : BM;
+    if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B)) return SQAP_ERR_CUDA;
+    if (!make_map(&tm_u, k.swiglu ? a.w_up : a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B))
+        return SQAP_ERR_CUDA;
+    if (!make_map(&tm_x, a.x8, a.M, a.K, k.BN / 2, BKH, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
+
     const int tiles = k.m_tiles * k.n_tiles;
     const int pairs = tiles < max_pairs ? tiles : max_pairs;
     w4a4_tc_pair_kernel<<<2 * pairs, THREADS, SMEM_BYTES, s>>>(tm_w, tm_u, tm_x, k);

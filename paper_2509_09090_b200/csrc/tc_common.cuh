@@ -218,6 +218,29 @@ inline bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t ro
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
 }
 
+// Splits M tokens into m_tiles tiles of BN tokens (multiple of 16, <= bn_max) for a persistent kernel whose
+// `units` workers (CTAs or CTA pairs) each take whole tiles: the split that minimises waves * (BN + overhead),
+// so that e.g. 224 tiles on 74 workers (4 waves, the last almost empty) become 288 narrower tiles (4 full waves).
+inline void choose_token_tiles(int M, int n_tiles, int units, int bn_max, int* m_tiles, int* BN) {
+    const int mt_min = (M + bn_max - 1) / bn_max;
+    *m_tiles = mt_min;
+    *BN = ((M + mt_min - 1) / mt_min + 15) / 16 * 16;
+    long best_cost = -1;
+    for (int mt = mt_min; mt <= mt_min + 12 && mt <= (M + 15) / 16; ++mt) {
+        const int per = (M + mt - 1) / mt;
+        const int bn = (per + 15) / 16 * 16;
+        if (bn > bn_max) continue;
+        const long tiles = static_cast<long>(mt) * n_tiles;
+        const long waves = (tiles + units - 1) / units;
+        const long cost = waves * (bn + 24);   // 24: per-tile overhead in token-equivalents
+        if (best_cost < 0 || cost < best_cost) {
+            best_cost = cost;
+            *m_tiles = mt;
+            *BN = bn;
+        }
+    }
+}
+
 inline int sm_count() {
     static int n = 0;
     if (!n) {
