@@ -304,7 +304,8 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
         if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
         *path = PATH_TC_PAIR;
     } else {
-        *path = a.M <= 8 ? PATH_GEMV : (tcgen05_supports(a) ? (a.M >= 512 ? PATH_TC_PAIR : PATH_TC) : PATH_SIMT);
+        // tensor-memory kernels: CTA pairs once there are enough token tiles to fill them, one CTA per tile below
+        *path = a.M <= 8 ? PATH_GEMV : (tcgen05_supports(a) ? (a.M >= 512 ? PATH_TC_PAIR : PATH_TC_TS) : PATH_SIMT);
     }
     return SQAP_OK;
 }
