@@ -309,17 +309,32 @@ def run_ours(args):
     if B.sqap_device_status() != B.SQAP_OK:
         raise SystemExit("bench.py: a kernel reported an expired bounded wait")
 
+    # The step's launches are recorded once into a CUDA graph and replayed: the same kernels, arguments and
+    # order as the eager calls above, without a host round trip per launch (--no-graph times the eager calls).
+    l0 = B.sqap_kernel_launch_count()
+    if args.no_graph:
+        step_fn = path.step
+        path.step()
+    else:
+        graph = torch.cuda.CUDAGraph()
+        with torch.cuda.graph(graph):
+            path.step()
+        step_fn = graph.replay
+    launches_per_step = B.sqap_kernel_launch_count() - l0
+    for _ in range(3):
+        step_fn()
+    torch.cuda.synchronize()
+
     sampler = ClockSampler(local_rank)
     if rank == 0:
         sampler.start()
-    l0 = B.sqap_kernel_launch_count()
-    ms = time_region(torch, path.step, args.steps, world)
-    launches = B.sqap_kernel_launch_count() - l0
+    ms = time_region(torch, step_fn, args.steps, world)
+    launches = launches_per_step * args.steps
     clocks = sampler.stop() if rank == 0 else None
 
     def e2e_step():
         path.upload()
-        path.step()
+        step_fn()
         path.download()
 
     for _ in range(2):
@@ -345,7 +360,7 @@ def run_ours(args):
             "tokens_per_s": world * M_FULL / (ms_step * 1e-3),
             "e2e": {"value": tops_e2e, "unit": "TOPS", "h2d_bytes_per_step": path.h2d_bytes,
                     "d2h_bytes_per_step": path.d2h_bytes, "tokens_per_s": world * M_FULL / (ms_e2e / args.steps * 1e-3)},
-            "gpu_launches": int(launches),
+            "gpu_launches": int(launches), "launch_mode": "eager" if args.no_graph else "cuda_graph replay",
             "clocks": clocks,
             "roofline": roof,
             "cpu_baseline": cpu,
@@ -582,10 +597,11 @@ def run_single_kernel(args):
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
-    ap.add_argument("--steps", type=int, default=20)
+    ap.add_argument("--steps", type=int, default=100)
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-graph", action="store_true", help="issue the step's launches eagerly instead of replaying a CUDA graph")
     ap.add_argument("--detail", action="store_true",
                     help="time every kernel of the path alone at the workload's shapes (one JSON table, no bench line)")
     ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "quantize", "prune"],
