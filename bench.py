@@ -242,8 +242,12 @@ def dominant_gemm_roofline(torch, B, path: Path, steps: int, peaks: dict):
     ops = 2.0 * M * N * K
     achieved = ops / (ms * 1e-3) / 1e12
     peak = 2.0 * peaks["bf16"]       # int8 dense = 2 x bf16 dense (nominal ratio) x the measured bf16 burst figure
-    return dict(bound="tensor", kernel="w4a4 linear GEMM, M=4608 N=12288 K=4096 (int8 MMA, int32 accumulate)",
-                achieved=achieved, peak=peak, unit="TOP/s", frac=achieved / peak, traffic=None,
+    # traffic: dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel at this shape, from the ncu
+    # capture summarised in profiles/w4a4_tc_pair_kernel_qkv_m4608.md (algorithmic bytes: 25.2 MB packed weights
+    # + 18.9 MB int8 activations + 113.2 MB fp16 output = 157.3 MB; part of the output is still in L2 at the end).
+    return dict(bound="tensor", kernel="w4a4_tc_pair_kernel: W4A4 linear GEMM, M=4608 N=12288 K=4096 (int8 MMA on CTA "
+                                       "pairs, int32 accumulate in tensor memory)",
+                achieved=achieved, peak=peak, unit="TOP/s", frac=achieved / peak, traffic=118.9e6,
                 peak_source=f"2 x bf16 burst ({peaks['source']})", ms_per_launch=ms)
 
 
