@@ -38,7 +38,8 @@ constexpr int WPH_BYTES = BM * BKH / 2;   // 8 KB: one half of a stage's packed 
 constexpr int OFF_X = 0;
 constexpr int OFF_WP = OFF_X + S * 2 * XH_BYTES;
 constexpr int OFF_BAR = OFF_WP + S * 2 * WPH_BYTES;
-constexpr int SMEM_BYTES = OFF_BAR + 512 + 1024;  // barriers + slack for 1024-byte alignment
+constexpr int OFF_TOK = OFF_BAR + 512;    // per-token epilogue constants, two tiles x BN_MAX x 8 bytes
+constexpr int SMEM_BYTES = OFF_TOK + 2 * BN_MAX * 8 + 1024;  // + slack for 1024-byte alignment
 constexpr int TMEM_A_COL = 2 * BN_MAX;    // columns [0,192) and [192,384): accumulators; from 384: weight tiles
 constexpr int A_COLS = BK / 4;            // 64 columns hold 256 int8 per lane
 constexpr int EPI_WARPS = 8;
@@ -240,7 +241,15 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
         for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x, ++lt) {
             const int b = lt & 1;
             const int n0 = (tile % a.n_tiles) * BM, m0 = (tile / a.n_tiles) * a.BN;
-            if (!__all_sync(0xffffffffu, mbar_wait(acc_full(b), (lt >> 1) & 1u, abort_flag))) { failed = true; break; }
+            // stage the tile's per-token constants (the other buffer may still be read by slower warps)
+            int2* tok = reinterpret_cast<int2*>(sm + OFF_TOK) + b * BN_MAX;
+            const int et = static_cast<int>(threadIdx.x) - 6 * 32;
+            if (et < a.BN) {
+                const int m = m0 + et;
+                tok[et] = m < a.M ? make_int2(__ldg(a.bias_sum + m) << 7, __float_as_int(__ldg(a.act_scales + m))) : make_int2(0, 0);
+            }
+            // all epilogue warps leave the loop together if any wait ran out, so the barrier below never hangs
+            if (bar_or(1, 32 * EPI_WARPS, !mbar_wait(acc_full(b), (lt >> 1) & 1u, abort_flag))) { failed = true; break; }
             tc_fence_after();
             const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(b * BN_MAX);
             int n;
@@ -256,12 +265,12 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
                 sw = n_ok ? __half2float(a.w_scales[n]) : 0.0f;
             }
             if (a.swiglu) {
-                if (a.out_dtype == SQAP_FP16) epilogue_tile<SQAP_FP16, true, 16>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
-                else epilogue_tile<SQAP_BF16, true, 16>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
+                if (a.out_dtype == SQAP_FP16) epilogue_tile_staged<SQAP_FP16, true, 16>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane, tok);
+                else epilogue_tile_staged<SQAP_BF16, true, 16>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane, tok);
             } else {
-                if (a.out_dtype == SQAP_FP16) epilogue_tile<SQAP_FP16, false>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
-                else if (a.out_dtype == SQAP_BF16) epilogue_tile<SQAP_BF16, false>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
-                else epilogue_tile<SQAP_I32, false>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane);
+                if (a.out_dtype == SQAP_FP16) epilogue_tile_staged<SQAP_FP16, false, 1>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane, tok);
+                else if (a.out_dtype == SQAP_BF16) epilogue_tile_staged<SQAP_BF16, false, 1>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane, tok);
+                else epilogue_tile_staged<SQAP_I32, false, 1>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane, tok);
             }
             tc_fence_before();
             __syncwarp();

@@ -183,6 +183,72 @@ __device__ __forceinline__ void epilogue_tile(const Args& a, uint32_t taddr, int
     }
 }
 
+// Barrier among `nthreads` threads (named barrier `id`) that also ORs a predicate over them: every thread gets
+// true if any thread passed true.
+__device__ __forceinline__ bool bar_or(int id, int nthreads, bool pred) {
+    uint32_t r;
+    asm volatile(
+        "{\n\t.reg .pred p, q;\n\t"
+        "setp.ne.b32 q, %3, 0;\n\t"
+        "bar.red.or.pred p, %1, %2, q;\n\t"
+        "selp.u32 %0, 1, 0, p;\n\t}"
+        : "=r"(r)
+        : "r"(id), "r"(nthreads), "r"(static_cast<uint32_t>(pred))
+        : "memory");
+    return r != 0;
+}
+
+// The same epilogue with the per-token constants staged in shared memory: tok[c] = {128 * bias_sum, bits of the
+// activation scale} of token m0 + c ({0, 0} past M). All lanes of a warp need the same token's pair, so one
+// broadcast shared-memory load per two tokens replaces four warp shuffles; the shuffles of the routine above
+// share a pipe with the unpack warps' shared-memory loads and were measured to slow the main loop.
+template <int OUT, bool SWIGLU, int XCHG>
+__device__ __forceinline__ void epilogue_tile_staged(const Args& a, uint32_t taddr, int m0, int c_begin, int c_end, int n,
+                                                     bool n_ok, float sw, int lane, const int2* tok) {
+    constexpr int ESZ = OUT == SQAP_I32 ? 4 : 2;
+    const bool odd = (lane & XCHG) != 0;   // SwiGLU: this lane holds the up projection, its partner (lane ^ XCHG) the gate
+    const int64_t row_bytes = a.ldo * ESZ;
+    for (int c = c_begin; c < c_end; c += 16) {
+        uint32_t v[16];
+        tc_ld16(taddr + c, v);
+        const int4* t4 = reinterpret_cast<const int4*>(tok + c);   // two tokens per 16-byte load
+        tc_wait_ld();
+        const int valid = a.M - (m0 + c);  // tokens of this chunk that exist
+        uint8_t* optr = static_cast<uint8_t*>(a.out) + static_cast<int64_t>(m0 + c) * row_bytes + static_cast<int64_t>(n) * ESZ;
+#pragma unroll
+        for (int j = 0; j < 16; j += 2) {
+            const int4 t = t4[j >> 1];
+            const int t0 = (static_cast<int>(v[j]) - t.x) >> 4, t1 = (static_cast<int>(v[j + 1]) - t.z) >> 4;
+            const float y0 = __fmul_rn(__fmul_rn(static_cast<float>(t0), __int_as_float(t.y)), sw);
+            const float y1 = __fmul_rn(__fmul_rn(static_cast<float>(t1), __int_as_float(t.w)), sw);
+            if (SWIGLU) {
+                // the gate lane finishes token j (needs the up value of its partner), the up lane token j+1
+                const float got = __shfl_xor_sync(0xffffffffu, odd ? y0 : y1, XCHG);
+                const float h = odd ? silu_mul_fast(got, y1) : silu_mul_fast(y0, got);
+                const int jj = odd ? j + 1 : j;
+                if (n_ok && jj < valid) {
+                    uint8_t* o = optr + jj * row_bytes;
+                    if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(h);
+                    else *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(h);
+                }
+            } else {
+                if (n_ok && j < valid) {
+                    uint8_t* o = optr + j * row_bytes;
+                    if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(y0);
+                    else if (OUT == SQAP_BF16) *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(y0);
+                    else *reinterpret_cast<int32_t*>(o) = t0;
+                }
+                if (n_ok && j + 1 < valid) {
+                    uint8_t* o = optr + (j + 1) * row_bytes;
+                    if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(y1);
+                    else if (OUT == SQAP_BF16) *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(y1);
+                    else *reinterpret_cast<int32_t*>(o) = t1;
+                }
+            }
+        }
+    }
+}
+
 // ------------------------------------------------------------------------------- host side
 typedef CUresult (*EncodeTiledFn)(CUtensorMap*, CUtensorMapDataType, cuuint32_t, void*, const cuuint64_t*,
                                   const cuuint64_t*, const cuuint32_t*, const cuuint32_t*, CUtensorMapInterleave,
