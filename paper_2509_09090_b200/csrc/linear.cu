@@ -235,6 +235,90 @@ __global__ void __launch_bounds__(256) w4a4_gemv_kernel(LinearArgs a) {
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Single-row decode step (M = 1): the one activation row lives in registers. A lane always meets the same
+// 16-byte weight chunks (lane, lane + 32, ...) of whatever row its warp streams, so it loads the 2 x 16
+// activation bytes that go with each of them once and then only streams weights: two rows at a time (all their
+// loads issued before the first dp4a), persistent warps striding over the output channels.
+template <bool SWIGLU, int CPL>
+__global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
+    const int lane = threadIdx.x & 31;
+    const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), W = gridDim.x * (blockDim.x >> 5);
+    const int chunks = a.K / 32;
+    uint4 xl[CPL], xh[CPL];
+#pragma unroll
+    for (int i = 0; i < CPL; ++i) {
+        const int c = lane + 32 * i;
+        xl[i] = xh[i] = make_uint4(0, 0, 0, 0);
+        if (c < chunks) {
+            int lo_k, hi_k;
+            chunk_k(c, a.half, lo_k, hi_k);
+            xl[i] = __ldg(reinterpret_cast<const uint4*>(a.x8 + lo_k));
+            xh[i] = __ldg(reinterpret_cast<const uint4*>(a.x8 + hi_k));
+        }
+    }
+    const int bs = a.bias_sum[0];
+    const float sx = a.act_scales[0];
+    auto dot = [&](const uint4* wv) {
+        int acc = 0;
+#pragma unroll
+        for (int i = 0; i < CPL; ++i) {
+            const uint32_t w4[4] = {wv[i].x, wv[i].y, wv[i].z, wv[i].w};
+            const int l4[4] = {(int)xl[i].x, (int)xl[i].y, (int)xl[i].z, (int)xl[i].w};
+            const int h4[4] = {(int)xh[i].x, (int)xh[i].y, (int)xh[i].z, (int)xh[i].w};
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                acc = __dp4a(l4[q], static_cast<int>(w4[q] & 0x0F0F0F0Fu), acc);
+                acc = __dp4a(h4[q], static_cast<int>(w4[q] & 0xF0F0F0F0u), acc);
+            }
+        }
+#pragma unroll
+        for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
+        return acc;
+    };
+    auto load_row = [&](const uint8_t* wbase, int n, uint4* wv) {
+        const uint4* row = reinterpret_cast<const uint4*>(wbase + static_cast<int64_t>(n) * (a.K / 2));
+#pragma unroll
+        for (int i = 0; i < CPL; ++i) {
+            const int c = lane + 32 * i;
+            wv[i] = c < chunks ? __ldg(row + c) : make_uint4(0, 0, 0, 0);   // zero weights meet zero activations
+        }
+    };
+    auto finish = [&](int n, int raw_g, int raw_u) {
+        if (lane != 0) return;
+        const int t = finish_acc(raw_g, bs);
+        float y = dequant(t, sx, __half2float(a.w_scales[n]));
+        if (SWIGLU) y = swiglu(y, dequant(finish_acc(raw_u, bs), sx, __half2float(a.w_up_scales[n])));
+        store_out(a.out, n, a.out_dtype, y, t);
+    };
+    constexpr bool TWO = !SWIGLU;   // rows in flight per warp (the gated pair already streams two weight rows)
+    for (int n = gw; n < a.N; n += (TWO ? 2 : 1) * W) {
+        const int n2 = n + W;
+        const bool two = TWO && n2 < a.N;
+        uint4 g0[CPL], g1[TWO ? CPL : 1], u0[SWIGLU ? CPL : 1];
+        load_row(a.w, n, g0);
+        if (SWIGLU) load_row(a.w_up, n, u0);
+        if (TWO && two) load_row(a.w, n2, g1);
+        finish(n, dot(g0), SWIGLU ? dot(u0) : 0);
+        if (TWO && two) finish(n2, dot(g1), 0);
+    }
+}
+
+template <int CPL>
+static void launch_gemv1(const LinearArgs& a, cudaStream_t s) {
+    static int blocks = 0;
+    if (!blocks) {
+        int dev = 0, sms = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        blocks = (sms > 0 ? sms : 148) * 3;
+    }
+    const int need = (a.N + 7) / 8;
+    const int grid = need < blocks ? need : blocks;
+    if (a.w_up) w4a4_gemv1_kernel<true, CPL><<<grid, 256, 0, s>>>(a);
+    else w4a4_gemv1_kernel<false, CPL><<<grid, 256, 0, s>>>(a);
+}
+
 template <int MM>
 static void launch_gemv(const LinearArgs& a, cudaStream_t s) {
     const int warps = 8;
@@ -305,7 +389,12 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
         *path = PATH_TC_PAIR;
     } else {
         // tensor-memory kernels: CTA pairs once there are enough token tiles to fill them, one CTA per tile below
-        *path = a.M <= 8 ? PATH_GEMV : (tcgen05_supports(a) ? (a.M >= 512 ? PATH_TC_PAIR : PATH_TC_TS) : PATH_SIMT);
+        // the weight-streaming kernel re-reads the activations per row of M, so beyond two rows it only wins where
+        // the tensor-memory kernel has too few weight tiles to fill the SMs
+        const bool tc_ok = tcgen05_supports(a);
+        const int w_tiles = (a.w_up ? 2 * a.N : a.N) / 128;
+        const bool gemv = a.M <= 8 && (!tc_ok || a.M <= 2 || (a.M <= 4 && w_tiles < 64));
+        *path = gemv ? PATH_GEMV : (tc_ok ? (a.M >= 512 ? PATH_TC_PAIR : PATH_TC_TS) : PATH_SIMT);
     }
     return SQAP_OK;
 }
@@ -315,7 +404,10 @@ static sqap_status run_gemm(const LinearArgs& a, LinearPath path, cudaStream_t s
     if (path == PATH_TC_TS) return launch_linear_tcgen05_ts(a, s);
     if (path == PATH_TC_PAIR) return launch_linear_tcgen05_pair(a, s);
     if (path == PATH_GEMV) {
-        if (a.M == 1) launch_gemv<1>(a, s);
+        const int chunks = a.K / 32;
+        // rows up to 4096 codes: activation row in registers; longer rows would not amortise loading it
+        if (a.M == 1 && chunks <= 32 * 4) launch_gemv1<4>(a, s);
+        else if (a.M == 1) launch_gemv<1>(a, s);
         else if (a.M == 2) launch_gemv<2>(a, s);
         else if (a.M <= 4) launch_gemv<4>(a, s);
         else launch_gemv<8>(a, s);
