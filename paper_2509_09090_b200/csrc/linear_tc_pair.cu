@@ -393,7 +393,7 @@ sqap_status launch_linear_tcgen05_pair(const LinearArgs& a, cudaStream_t s) {
         }
         max_pairs = n;
     }
-    choose_token_tiles(a.M, k.n_tiles, max_pairs, BN_MAX, &k.m_tiles, &k.BN);
+    choose_token_tiles(a.M, k.n_tiles, max_pairs, BN_MAX, 128, &k.m_tiles, &k.BN);
     CUtensorMap tm_w, tm_u, tm_x;
     const uint32_t w_box_rows = k.swiglu ? BM / 2 : BM;
     if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B)) return SQAP_ERR_CUDA;

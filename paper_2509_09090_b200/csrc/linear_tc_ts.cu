@@ -306,7 +306,7 @@ sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s) {
     k.K = a.K;
     k.swiglu = a.w_up ? 1 : 0;
     k.n_tiles = k.swiglu ? (2 * a.N + BM - 1) / BM : (a.N + BM - 1) / BM;
-    choose_token_tiles(a.M, k.n_tiles, sm_count(), BN_MAX, &k.m_tiles, &k.BN);
+    choose_token_tiles(a.M, k.n_tiles, sm_count(), BN_MAX, 256, &k.m_tiles, &k.BN);
     k.out_dtype = a.out_dtype;
     k.status = device_status_word();
     if (!k.status) return SQAP_ERR_CUDA;

@@ -285,20 +285,24 @@ inline bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t ro
 }
 
 // Splits M tokens into m_tiles tiles of BN tokens (multiple of 16, <= bn_max) for a persistent kernel whose
-// `units` workers (CTAs or CTA pairs) each take whole tiles: the split that minimises waves * (BN + overhead),
-// so that e.g. 224 tiles on 74 workers (4 waves, the last almost empty) become 288 narrower tiles (4 full waves).
-inline void choose_token_tiles(int M, int n_tiles, int units, int bn_max, int* m_tiles, int* BN) {
+// `units` workers (CTAs or CTA pairs) each take whole tiles: the split that minimises waves x time per tile, so
+// that e.g. 224 tiles on 74 workers (4 waves, the last almost empty) become 288 narrower tiles (4 full waves).
+// Time per 256-code stage of a tile, in cycles: the MMAs take 4 per token, the stage's TMA traffic (16 KB of
+// packed weights + x_bytes_per_token per token: 256, or 128 where a CTA pair shares the token tile) moves at
+// about 58 bytes per cycle, and each tile costs about 96 more per stage for its fill and hand-over.
+inline void choose_token_tiles(int M, int n_tiles, int units, int bn_max, int x_bytes_per_token, int* m_tiles, int* BN) {
     const int mt_min = (M + bn_max - 1) / bn_max;
     *m_tiles = mt_min;
     *BN = ((M + mt_min - 1) / mt_min + 15) / 16 * 16;
-    long best_cost = -1;
+    double best_cost = -1.0;
     for (int mt = mt_min; mt <= mt_min + 12 && mt <= (M + 15) / 16; ++mt) {
         const int per = (M + mt - 1) / mt;
         const int bn = (per + 15) / 16 * 16;
         if (bn > bn_max) continue;
         const long tiles = static_cast<long>(mt) * n_tiles;
         const long waves = (tiles + units - 1) / units;
-        const long cost = waves * (bn + 24);   // 24: per-tile overhead in token-equivalents
+        const double mma = 4.0 * bn, fetch = (16384.0 + static_cast<double>(x_bytes_per_token) * bn) / 58.0;
+        const double cost = static_cast<double>(waves) * ((mma > fetch ? mma : fetch) + 96.0);
         if (best_cost < 0 || cost < best_cost) {
             best_cost = cost;
             *m_tiles = mt;
