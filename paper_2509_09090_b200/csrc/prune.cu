@@ -29,8 +29,18 @@ __global__ void __launch_bounds__(512) prune_select_kernel(sqap_prune_params p, 
         float s;
         if (p.score_rows > 0) {
             const __half* A = static_cast<const __half*>(scores) + static_cast<int64_t>(b) * p.score_rows * nv;
+            // batches of 8 loads in flight (the rows are nv apart: every load is a separate L2 access), summed in
+            // row order
             s = __half2float(A[j]);
-            for (int r = 1; r < p.score_rows; ++r) s = __fadd_rn(s, __half2float(A[static_cast<int64_t>(r) * nv + j]));
+            int r = 1;
+            for (; r + 8 <= p.score_rows; r += 8) {
+                __half h[8];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) h[i] = A[static_cast<int64_t>(r + i) * nv + j];
+#pragma unroll
+                for (int i = 0; i < 8; ++i) s = __fadd_rn(s, __half2float(h[i]));
+            }
+            for (; r < p.score_rows; ++r) s = __fadd_rn(s, __half2float(A[static_cast<int64_t>(r) * nv + j]));
         } else {
             s = static_cast<const float*>(scores)[static_cast<int64_t>(b) * nv + j];
         }
