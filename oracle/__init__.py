@@ -107,6 +107,18 @@ def rotate_rows(x_bits, rotate=True):
     return out
 
 
+def quantize_weights(w_bits, rotate=False):
+    """w_bits: uint16 view of fp16 [N, K]. Returns (codes i8 [N,K], scales fp16 bits u16 [N])."""
+    w = _c(w_bits, np.uint16)
+    N, K = w.shape
+    codes = np.empty((N, K), np.int8)
+    scales = np.empty((N,), np.uint16)
+    rc = lib().oracle_quantize_weights(_p(w), N, K, ctypes.c_int64(K), int(rotate), _p(codes), _p(scales))
+    if rc != 0:
+        raise ValueError(f"oracle_quantize_weights: {rc}")
+    return codes, scales
+
+
 def quantize_act(x_bits, rotate=False, row_index=None, ldx=None, K=None):
     """x_bits: uint16 view of fp16 [rows, ldx]. Returns (packed u8 [M,K/2], scales f32 [M], codes i8 [M,K])."""
     x = _c(x_bits, np.uint16)

@@ -236,6 +236,63 @@ void oracle_rotate_rows(const uint16_t *x, int M, int K, int64_t ldx, int rotate
     }
 }
 
+/* ---------------------------------------------------------------- offline weight quantizer */
+
+/*
+ * Offline side of W4A4 ("4-bit weights"; Eq. 6 for rotated layers): per-output-channel symmetric
+ * round-to-nearest INT4 quantization of an fp16 weight matrix W [N][K] (row n = output channel n).
+ *   v     = fp32(W[n])                 [rotate: v = FWHT(v) * (1/sqrt K), i.e. row n of W H^T; the
+ *                                        Sylvester matrix is symmetric, so H applied to the row is that]
+ *   amax  = max |v|
+ *   amax==0 : scale = fp16(1), codes 0
+ *   else    : s16 = fp16_rn(amax / 7), raised to the smallest positive fp16 if that rounds to zero
+ *   sf    = fp32(s16)
+ *   q     = clamp( rint(v / sf), -8, 7 )              (fp32 division, ties to even)
+ * The scale is rounded to fp16 BEFORE the codes are taken, because fp16 is what the linear
+ * multiplies with. Returns 0, -1 on bad arguments, -3 if a scale is not finite.
+ */
+int oracle_quantize_weights(const uint16_t *w, int N, int K, int64_t ldw, int rotate, int8_t *codes,
+                            uint16_t *scales_fp16)
+{
+    if (N < 0 || K <= 0) return -1;
+    if (rotate && (K & (K - 1))) return -1;
+    const float norm = oracle_hadamard_norm(K);
+    int err = 0;
+#pragma omp parallel for schedule(static)
+    for (int n = 0; n < N; ++n) {
+        float *v = (float *)malloc(sizeof(float) * (size_t)K);
+        if (!v) { err = 1; continue; }
+        for (int k = 0; k < K; ++k) v[k] = half_bits_to_float(w[(int64_t)n * ldw + k]);
+        if (rotate) {
+            oracle_fwht_f32(v, K);
+            for (int k = 0; k < K; ++k) v[k] = v[k] * norm;
+        }
+        float amax = 0.0f;
+        for (int k = 0; k < K; ++k) {
+            float a = fabsf(v[k]);
+            if (a > amax) amax = a;
+        }
+        uint16_t s16;
+        if (amax == 0.0f) {
+            s16 = 0x3C00; /* 1.0 */
+        } else {
+            s16 = float_to_half_bits(amax / 7.0f);
+            if ((s16 & 0x7FFF) == 0) s16 = 0x0001;
+            if ((s16 & 0x7C00) == 0x7C00) err = 3; /* inf / nan: weights out of the fp16 range of scales */
+        }
+        scales_fp16[n] = s16;
+        const float sf = half_bits_to_float(s16);
+        for (int k = 0; k < K; ++k) {
+            int q = (int)rintf(v[k] / sf);
+            if (q < -8) q = -8;
+            if (q > 7) q = 7;
+            codes[(int64_t)n * K + k] = (int8_t)q;
+        }
+        free(v);
+    }
+    return err == 1 ? -2 : (err == 3 ? -3 : 0);
+}
+
 /* Two's-complement nibble pairs -> int8 codes (even index in the low nibble). */
 void oracle_unpack_nibbles(const uint8_t *packed, int64_t n_codes, int8_t *codes)
 {

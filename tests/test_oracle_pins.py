@@ -212,6 +212,80 @@ def test_quantizer_row_index_and_stride():
     assert np.array_equal(p3, p4) and np.array_equal(s3, s4)
 
 
+# ------------------------------------------------------------------ offline weight quantizer
+
+def _fp16_weights(seed, N, K, outlier_cols=0):
+    w = (wl.activations(seed, 9, N, K, outlier_cols, 25.0).astype(np.float32) * np.float32(0.02)).astype(np.float16)
+    return w
+
+
+@pytest.mark.parametrize("rotate", [False, True])
+def test_weight_quantizer_scale_error_bound_and_exact_rounding(rotate):
+    """Per-channel RTN: the scale is numpy's own fp16 rounding of amax/7, every code is the nearest integer of
+    v / scale (exact rational arithmetic away from ties), and the dequantised error is at most half a scale."""
+    N, K = 24, 256
+    w = _fp16_weights(31, N, K, outlier_cols=3)
+    w[5] = 0
+    codes, s_bits = oracle.quantize_weights(bits(w), rotate=rotate)
+    v = oracle.rotate_rows(bits(w), rotate=rotate)                      # the fp32 rows the quantizer sees
+    amax = np.abs(v).max(axis=1)
+    s_np = (amax / np.float32(7.0)).astype(np.float16)                  # independent fp16 rounding
+    s_np[amax == 0] = np.float16(1.0)
+    assert np.array_equal(s_bits.view(np.float16), s_np)
+    sf = s_bits.view(np.float16).astype(np.float64)
+    assert codes.min() >= -7 and codes.max() <= 7                       # fp16 rounding moves v/s by < 2^-10: no clamp
+    err = np.abs(v.astype(np.float64) - sf[:, None] * codes)
+    assert (err <= sf[:, None] / 2 * (1 + 2.0 ** -20)).all()
+    assert not codes[5].any()
+    undecided = 0
+    for n in range(0, N, 5):
+        if amax[n] == 0:
+            continue
+        sfr = Fraction(float(sf[n]))
+        for k in range(K):
+            r = Fraction(float(v[n, k])) / sfr
+            fl = math.floor(r)
+            frac = r - fl
+            if abs(frac - Fraction(1, 2)) < Fraction(1, 2 ** 19):
+                undecided += 1
+                continue
+            assert codes[n, k] == fl + (1 if frac > Fraction(1, 2) else 0), (n, k)
+    assert undecided < 10
+
+
+def test_weight_quantizer_ties_scaling_and_tiny_rows():
+    row = np.array([7, 0.5, 1.5, 2.5, -0.5, -1.5, -2.5, 3.5, -3.5, 6.5, -6.5, 0, 0.25, -0.75, 4.5, 5.5], np.float16)
+    codes, s = oracle.quantize_weights(bits(np.stack([row, row * np.float16(4)])))
+    assert codes[0].tolist() == [7, 0, 2, 2, 0, -2, -2, 4, -4, 6, -6, 0, 0, -1, 4, 6]    # scale exactly 1: ties to even
+    assert s.view(np.float16).tolist() == [1.0, 4.0] and np.array_equal(codes[0], codes[1])  # power-of-two invariance
+    tiny = np.zeros((1, 32), np.float16)
+    tiny[0, 3] = np.float16(2.0 ** -24)                                  # amax/7 underflows fp16: smallest scale used
+    codes, s = oracle.quantize_weights(bits(tiny))
+    assert s[0] == 1 and codes[0, 3] == 1 and np.count_nonzero(codes) == 1
+
+
+def test_eq6_rotated_w4a4_product_approximates_the_fp_product():
+    """Eq. 6 end to end on the oracle: quantizing W H^T and H x and multiplying the codes approximates W x, the
+    rotation changes nothing in exact arithmetic (checked in fp64 on the unquantized rows), and with outlier
+    channels the rotated product is the more accurate one (the reason the paper rotates)."""
+    N, K, M = 32, 512, 16
+    w = _fp16_weights(33, N, K)
+    x = wl.activations(34, 2, M, K, 6, 30.0)
+    ref = x.astype(np.float64) @ w.astype(np.float64).T
+    # exactness of the rotation itself
+    hw = oracle.rotate_rows(bits(w), rotate=True).astype(np.float64)
+    hx = oracle.rotate_rows(bits(x), rotate=True).astype(np.float64)
+    assert np.allclose(hx @ hw.T, ref, rtol=0, atol=1e-3 * np.abs(ref).max())
+    errs = {}
+    for rot in (False, True):
+        wc, ws = oracle.quantize_weights(bits(w), rotate=rot)
+        _, sx, xc = oracle.quantize_act(bits(x), rotate=rot)
+        acc = oracle.gemm_i32(xc, wc).astype(np.float64)
+        y = acc * sx[:, None].astype(np.float64) * ws.view(np.float16).astype(np.float64)[None, :]
+        errs[rot] = np.sqrt(np.mean((y - ref) ** 2)) / np.sqrt(np.mean(ref ** 2))
+    assert errs[True] < 0.25 and errs[True] < 0.6 * errs[False], errs
+
+
 def test_pack_unpack_round_trip_all_pairs():
     a, b = np.meshgrid(np.arange(-8, 8), np.arange(-8, 8))
     codes = np.stack([a.ravel(), b.ravel()], axis=1).astype(np.int8)
