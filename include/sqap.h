@@ -79,6 +79,21 @@ typedef struct sqap_weights sqap_weights;
 sqap_status sqap_pack_weights(const int8_t* codes, const uint16_t* scales_fp16, int N, int K, uint32_t flags,
                               void* stream, sqap_weights** out);
 
+/*
+ * Offline weight quantizer ("4-bit weights", per-output-channel symmetric round-to-nearest; with
+ * SQAP_Q_ROTATE the weight side of Eq. 6: the codes are those of W H^T, H = Sylvester-Hadamard / sqrt(K),
+ * to be multiplied with activations quantized with SQAP_Q_ROTATE). For every output channel n:
+ *   v = fp32(W[n])  [rotated: H v] ; amax = max|v|
+ *   scale = fp16(amax / 7)  (fp16(1) for an all-zero row; the smallest positive fp16 if that underflows)
+ *   code  = clamp(round_half_even(v / fp32(scale)), -8, 7)
+ * w_fp16: device fp16 [N rows, ldw elements apart]; codes_out: device int8 [N*K]; scales_out_fp16: device [N].
+ * K % 32 == 0, K <= 32768; rotation needs K a power of two >= 64. The outputs are what sqap_pack_weights takes
+ * (pass SQAP_W_ROTATED there for rotated weights). Weights whose amax / 7 exceeds the fp16 range give an
+ * infinite scale, which sqap_pack_weights rejects (SQAP_ERR_RANGE). Enqueues on `stream`, does not synchronise.
+ */
+sqap_status sqap_quantize_weights(const void* w_fp16, int N, int K, int64_t ldw, uint32_t flags, int8_t* codes_out,
+                                  uint16_t* scales_out_fp16, void* stream);
+
 /* Releases a handle (NULL is accepted). Synchronises the device. */
 sqap_status sqap_free_weights(sqap_weights* w);
 

@@ -54,6 +54,56 @@ __global__ void unpack_weights_kernel(const uint8_t* __restrict__ packed, int N,
     }
 }
 
+// ---------------------------------------------------------------------------------------------
+// Offline weight quantizer: fp16 W [N][K] -> INT4 codes + fp16 per-channel scales, with the optional
+// rotation of Eq. 6 (row n of W H^T = H applied to row n; H symmetric). Offline and run once per model,
+// so it is written for clarity: one CTA per output channel, the row in shared memory as fp32, the
+// Walsh-Hadamard stages h = 1, 2, 4, ... applied one after the other with a barrier between them
+// (every stage output is one fp32 add of two fixed inputs, so the bits do not depend on the thread map).
+__global__ void __launch_bounds__(256) quantize_weight_rows_kernel(const __half* __restrict__ w, int K, int64_t ldw,
+                                                                   int rotate, float norm, int8_t* __restrict__ codes,
+                                                                   __half* __restrict__ scales) {
+    extern __shared__ float row[];   // K floats
+    __shared__ float red[8];
+    const int n = blockIdx.x;
+    const __half* wr = w + static_cast<int64_t>(n) * ldw;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) row[k] = __half2float(wr[k]);
+    __syncthreads();
+    if (rotate) {
+        for (int h = 1; h < K; h <<= 1) {
+            for (int pr = threadIdx.x; pr < K / 2; pr += blockDim.x) {
+                const int j = (pr / h) * 2 * h + (pr % h);
+                const float a = row[j], b = row[j + h];
+                row[j] = __fadd_rn(a, b);
+                row[j + h] = __fsub_rn(a, b);
+            }
+            __syncthreads();
+        }
+        for (int k = threadIdx.x; k < K; k += blockDim.x) row[k] = __fmul_rn(row[k], norm);
+        __syncthreads();
+    }
+    float amax = 0.0f;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) amax = fmaxf(amax, fabsf(row[k]));
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) amax = fmaxf(amax, __shfl_xor_sync(0xffffffffu, amax, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = amax;
+    __syncthreads();
+    amax = red[0];
+    for (int i = 1; i < (blockDim.x >> 5); ++i) amax = fmaxf(amax, red[i]);
+    __half s16 = __float2half_rn(1.0f);
+    if (amax != 0.0f) {
+        s16 = __float2half_rn(__fdiv_rn(amax, 7.0f));
+        if ((__half_as_ushort(s16) & 0x7FFF) == 0) s16 = __ushort_as_half(0x0001);   // smallest positive fp16
+    }
+    if (threadIdx.x == 0) scales[n] = s16;
+    const float sf = __half2float(s16);
+    int8_t* cr = codes + static_cast<int64_t>(n) * K;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        const int q = __float2int_rn(__fdiv_rn(row[k], sf));
+        cr[k] = static_cast<int8_t>(max(-8, min(7, q)));
+    }
+}
+
 static bool is_device_pointer(const void* p) {
     cudaPointerAttributes a;
     if (cudaPointerGetAttributes(&a, p) != cudaSuccess) {
@@ -140,6 +190,34 @@ fail:
     cudaFree(w->scales);
     delete w;
     return st;
+}
+
+sqap_status sqap_quantize_weights(const void* w_fp16, int N, int K, int64_t ldw, uint32_t flags, int8_t* codes_out,
+                                  uint16_t* scales_out_fp16, void* stream) {
+    using namespace sqap;
+    if (N < 0 || K <= 0 || ldw < K) return SQAP_ERR_INVALID;
+    if (flags & ~SQAP_Q_ROTATE) return SQAP_ERR_INVALID;
+    if (N == 0) return SQAP_OK;
+    if (!w_fp16 || !codes_out || !scales_out_fp16) return SQAP_ERR_INVALID;
+    if (K % 32 != 0) return SQAP_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(w_fp16) & 1u) || (reinterpret_cast<uintptr_t>(scales_out_fp16) & 1u)) return SQAP_ERR_ALIGN;
+    const bool rotate = (flags & SQAP_Q_ROTATE) != 0;
+    if (rotate && ((K & (K - 1)) != 0 || K < 64)) return SQAP_ERR_UNSUPPORTED;
+    if (K > 32768) return SQAP_ERR_UNSUPPORTED;   // the row is held in shared memory as fp32
+    const size_t smem = sizeof(float) * static_cast<size_t>(K);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(quantize_weight_rows_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem));
+        if (e != cudaSuccess) {
+            note_cuda_error(e);
+            return SQAP_ERR_CUDA;
+        }
+    }
+    const float norm = static_cast<float>(1.0 / sqrt(static_cast<double>(K)));
+    quantize_weight_rows_kernel<<<N, 256, smem, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const __half*>(w_fp16), K, ldw, rotate ? 1 : 0, norm, codes_out, reinterpret_cast<__half*>(scales_out_fp16));
+    count_launch();
+    return check_launch();
 }
 
 sqap_status sqap_free_weights(sqap_weights* w) {

@@ -169,6 +169,48 @@ def test_pack_rejects_bad_codes_and_scales():
     assert e.value.status == B.SQAP_ERR_ALIGN
 
 
+@pytest.mark.parametrize("N,K,rotate", [(24, 256, False), (24, 256, True), (130, 4096, True), (9, 11008, False),
+                                        (3, 64, True), (5, 16384, True), (40, 96, False)])
+def test_weight_quantizer_bit_exact_and_feeds_the_linear(N, K, rotate):
+    """sqap_quantize_weights against the oracle (codes and fp16 scale bits), then the quantized weights through
+    pack + linear against the oracle's integer GEMM on the same codes."""
+    w = (wl.activations(41, N + K, N, K, max(1, K // 100), 25.0).astype(np.float32) * np.float32(0.02)).astype(np.float16)
+    w[N // 2] = 0
+    wd = G.to_dev(w)
+    codes = torch.empty(N, K, dtype=torch.int8, device="cuda")
+    scales = torch.empty(N, dtype=torch.float16, device="cuda")
+    B.sqap_quantize_weights(wd, N, K, K, B.SQAP_Q_ROTATE if rotate else 0, codes, scales)
+    torch.cuda.synchronize()
+    co, so = oracle.quantize_weights(bits(w), rotate=rotate)
+    assert np.array_equal(codes.cpu().numpy(), co)
+    assert np.array_equal(scales.cpu().numpy().view(np.uint16), so)
+    if rotate or K % 32 == 0:
+        x = wl.activations(42, K, 20, K, max(1, K // 100), 30.0)
+        handle = B.sqap_pack_weights(codes, scales, N, K, B.SQAP_W_ROTATED if rotate else 0)   # device pointers
+        torch.cuda.synchronize()
+        _, sx, xc = oracle.quantize_act(bits(x), rotate=rotate)
+        acc = G.quantize_linear(x, handle, rotate=rotate, out_dtype=B.SQAP_I32)
+        assert np.array_equal(acc, oracle.gemm_i32(xc, co))
+        out = G.quantize_linear(x, handle, rotate=rotate)
+        ref = oracle.epilogue(oracle.gemm_i32(xc, co), sx, so)
+        assert G.within_tolerance(out, ref).all()
+        handle.close()
+
+
+def test_weight_quantizer_rejects_bad_arguments():
+    w = torch.zeros(8 * 96, dtype=torch.float16, device="cuda")
+    c = torch.zeros(8 * 96, dtype=torch.int8, device="cuda")
+    s = torch.zeros(8, dtype=torch.float16, device="cuda")
+    L = B.lib()
+    st = lambda *a: L.sqap_quantize_weights(*a, None)
+    assert st(w.data_ptr(), -1, 96, 96, 0, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
+    assert st(w.data_ptr(), 8, 96, 64, 0, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
+    assert st(w.data_ptr(), 8, 48, 48, 0, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_ALIGN
+    assert st(w.data_ptr(), 8, 96, 96, B.SQAP_Q_ROTATE, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_UNSUPPORTED
+    assert st(None, 8, 96, 96, 0, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
+    assert st(w.data_ptr(), 0, 96, 96, 0, None, None) == B.SQAP_OK
+
+
 # ------------------------------------------------------------------ linear: small and ragged shapes
 
 @pytest.mark.parametrize("M,N,K", [(1, 8, 32), (2, 128, 64), (7, 8, 512), (64, 512, 512), (65, 130, 96),
