@@ -107,20 +107,22 @@ def rotate_rows(x_bits, rotate=True):
     return out
 
 
-def quantize_weights(w_bits, rotate=False):
-    """w_bits: uint16 view of fp16 [N, K]. Returns (codes i8 [N,K], scales fp16 bits u16 [N])."""
+def quantize_weights(w_bits, rotate=False, ch_mul=None):
+    """w_bits: uint16 view of fp16 [N, K]; ch_mul: fp32 [K] or None. Returns (codes i8 [N,K], scales fp16 bits u16 [N])."""
     w = _c(w_bits, np.uint16)
     N, K = w.shape
     codes = np.empty((N, K), np.int8)
     scales = np.empty((N,), np.uint16)
-    rc = lib().oracle_quantize_weights(_p(w), N, K, ctypes.c_int64(K), int(rotate), _p(codes), _p(scales))
+    cm = _c(ch_mul, np.float32) if ch_mul is not None else None
+    rc = lib().oracle_quantize_weights(_p(w), N, K, ctypes.c_int64(K), int(rotate), _p(cm), _p(codes), _p(scales))
     if rc != 0:
         raise ValueError(f"oracle_quantize_weights: {rc}")
     return codes, scales
 
 
-def quantize_act(x_bits, rotate=False, row_index=None, ldx=None, K=None):
-    """x_bits: uint16 view of fp16 [rows, ldx]. Returns (packed u8 [M,K/2], scales f32 [M], codes i8 [M,K])."""
+def quantize_act(x_bits, rotate=False, row_index=None, ldx=None, K=None, per_tensor=False, ch_mul=None):
+    """x_bits: uint16 view of fp16 [rows, ldx]. Returns (packed u8 [M,K/2], scales f32 [M], codes i8 [M,K]).
+    per_tensor: one scale over all rows; ch_mul: fp32 [K] channel multiplier applied first."""
     x = _c(x_bits, np.uint16)
     if ldx is None:
         ldx = x.shape[1]
@@ -134,8 +136,13 @@ def quantize_act(x_bits, rotate=False, row_index=None, ldx=None, K=None):
     packed = np.empty((M, K // 2), np.uint8)
     scales = np.empty((M,), np.float32)
     codes = np.empty((M, K), np.int8)
-    rc = lib().oracle_quantize_act(_p(x), M, K, ctypes.c_int64(ldx), _p(row_index), int(rotate), _p(packed),
-                                   _p(scales), _p(codes))
+    cm = _c(ch_mul, np.float32) if ch_mul is not None else None
+    if per_tensor or cm is not None:
+        rc = lib().oracle_quantize_act_ex(_p(x), M, K, ctypes.c_int64(ldx), _p(row_index), int(rotate), int(per_tensor),
+                                          _p(cm), _p(packed), _p(scales), _p(codes))
+    else:
+        rc = lib().oracle_quantize_act(_p(x), M, K, ctypes.c_int64(ldx), _p(row_index), int(rotate), _p(packed),
+                                       _p(scales), _p(codes))
     if rc != 0:
         raise ValueError(f"oracle_quantize_act: bad arguments ({rc})")
     return packed, scales, codes

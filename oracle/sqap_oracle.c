@@ -158,41 +158,73 @@ float oracle_hadamard_norm(int K) { return (float)(1.0 / sqrt((double)K)); }
 /* ---------------------------------------------------------------- activation quantizer */
 
 /*
- * Per-token symmetric INT4 quantization of fp16 activations (Sec. "Pruning-Targeted
- * Quantizer Enhancement"; 4-bit activations of the W4A4 model), with the optional Hadamard
- * rotation of Eq. 6 applied to the row first.
+ * Symmetric INT4 quantization of fp16 activations (Sec. "Pruning-Targeted Quantizer Enhancement";
+ * 4-bit activations of the W4A4 model), with the optional Hadamard rotation of Eq. 6 applied to
+ * the row first, in the three granularities the paper names:
+ *   per token   (the default; one scale per row)
+ *   per tensor  ("tensor-wise quantization", Sec. 2.2 / 3): one scale from the amax over ALL rows,
+ *               reported in every scales[i]
+ *   per channel ("channel-wise quantization for activations", Sec. 3.3), read as a static
+ *               multiplier m[k] per input channel applied before anything else (smoothing); the
+ *               reciprocal belongs into the weights (oracle_quantize_weights takes it)
  *
  * Row i reads x[src*ldx .. +K) with src = row_index ? row_index[i] : i.
- *   v       = fp32(x)                        [rotate: v = FWHT(v) * (1/sqrt K)]
- *   amax    = max |v|
+ *   v       = fp32(x)                        [ch_mul: v[k] = v[k] * m[k], one fp32 multiply]
+ *                                            [rotate: v = FWHT(v) * (1/sqrt K)]
+ *   amax    = max |v|  over the row, or over all M rows (per_tensor)
  *   amax==0 : scale 1, all codes 0
  *   else    : scale = amax / 7 ; inv = 7 / amax           (two fp32 divisions)
  *   q       = clamp( rint(v * inv), -8, 7 )               (fp32 multiply, ties to even)
  *   packed byte j = (q[2j] & 15) | (q[2j+1] & 15) << 4
  * Returns 0, or -1 on bad arguments.
  */
-int oracle_quantize_act(const uint16_t *x, int M, int K, int64_t ldx, const int32_t *row_index,
-                        int rotate, uint8_t *q_packed, float *scales, int8_t *codes_out /* nullable [M*K] */)
+static void act_row(const uint16_t *xr, int K, int rotate, const float *ch_mul, float norm, float *v)
+{
+    for (int k = 0; k < K; ++k) v[k] = half_bits_to_float(xr[k]);
+    if (ch_mul)
+        for (int k = 0; k < K; ++k) v[k] = v[k] * ch_mul[k];
+    if (rotate) {
+        oracle_fwht_f32(v, K);
+        for (int k = 0; k < K; ++k) v[k] = v[k] * norm;
+    }
+}
+
+int oracle_quantize_act_ex(const uint16_t *x, int M, int K, int64_t ldx, const int32_t *row_index,
+                           int rotate, int per_tensor, const float *ch_mul, uint8_t *q_packed, float *scales,
+                           int8_t *codes_out /* nullable [M*K] */)
 {
     if (M < 0 || K <= 0 || (K & 1)) return -1;
     if (rotate && (K & (K - 1))) return -1;
     const float norm = oracle_hadamard_norm(K);
     int err = 0;
+    float tensor_amax = 0.0f;
+    if (per_tensor) {
+        float *v = (float *)malloc(sizeof(float) * (size_t)K);
+        if (!v) return -2;
+        for (int i = 0; i < M; ++i) {
+            int64_t src = row_index ? (int64_t)row_index[i] : (int64_t)i;
+            act_row(x + src * ldx, K, rotate, ch_mul, norm, v);
+            for (int k = 0; k < K; ++k) {
+                float a = fabsf(v[k]);
+                if (a > tensor_amax) tensor_amax = a;
+            }
+        }
+        free(v);
+    }
 #pragma omp parallel for schedule(static)
     for (int i = 0; i < M; ++i) {
         float *v = (float *)malloc(sizeof(float) * (size_t)K);
         if (!v) { err = 1; continue; }
         int64_t src = row_index ? (int64_t)row_index[i] : (int64_t)i;
-        const uint16_t *xr = x + src * ldx;
-        for (int k = 0; k < K; ++k) v[k] = half_bits_to_float(xr[k]);
-        if (rotate) {
-            oracle_fwht_f32(v, K);
-            for (int k = 0; k < K; ++k) v[k] = v[k] * norm;
-        }
+        act_row(x + src * ldx, K, rotate, ch_mul, norm, v);
         float amax = 0.0f;
-        for (int k = 0; k < K; ++k) {
-            float a = fabsf(v[k]);
-            if (a > amax) amax = a;
+        if (per_tensor) {
+            amax = tensor_amax;
+        } else {
+            for (int k = 0; k < K; ++k) {
+                float a = fabsf(v[k]);
+                if (a > amax) amax = a;
+            }
         }
         float scale, inv;
         if (amax == 0.0f) {
@@ -222,6 +254,13 @@ int oracle_quantize_act(const uint16_t *x, int M, int K, int64_t ldx, const int3
     return err ? -2 : 0;
 }
 
+/* The per-token quantizer without smoothing: the form the hot path uses. */
+int oracle_quantize_act(const uint16_t *x, int M, int K, int64_t ldx, const int32_t *row_index,
+                        int rotate, uint8_t *q_packed, float *scales, int8_t *codes_out /* nullable [M*K] */)
+{
+    return oracle_quantize_act_ex(x, M, K, ldx, row_index, rotate, 0, NULL, q_packed, scales, codes_out);
+}
+
 /* The rotated (or plain) fp32 row the quantizer sees, exposed for the pins. */
 void oracle_rotate_rows(const uint16_t *x, int M, int K, int64_t ldx, int rotate, float *out)
 {
@@ -241,7 +280,9 @@ void oracle_rotate_rows(const uint16_t *x, int M, int K, int64_t ldx, int rotate
 /*
  * Offline side of W4A4 ("4-bit weights"; Eq. 6 for rotated layers): per-output-channel symmetric
  * round-to-nearest INT4 quantization of an fp16 weight matrix W [N][K] (row n = output channel n).
- *   v     = fp32(W[n])                 [rotate: v = FWHT(v) * (1/sqrt K), i.e. row n of W H^T; the
+ *   v     = fp32(W[n])                 [ch_mul: v[k] = v[k] * d[k], the reciprocal of the activation
+ *                                        side's channel multiplier, one fp32 multiply]
+ *                                      [rotate: v = FWHT(v) * (1/sqrt K), i.e. row n of W H^T; the
  *                                        Sylvester matrix is symmetric, so H applied to the row is that]
  *   amax  = max |v|
  *   amax==0 : scale = fp16(1), codes 0
@@ -251,8 +292,8 @@ void oracle_rotate_rows(const uint16_t *x, int M, int K, int64_t ldx, int rotate
  * The scale is rounded to fp16 BEFORE the codes are taken, because fp16 is what the linear
  * multiplies with. Returns 0, -1 on bad arguments, -3 if a scale is not finite.
  */
-int oracle_quantize_weights(const uint16_t *w, int N, int K, int64_t ldw, int rotate, int8_t *codes,
-                            uint16_t *scales_fp16)
+int oracle_quantize_weights(const uint16_t *w, int N, int K, int64_t ldw, int rotate, const float *ch_mul,
+                            int8_t *codes, uint16_t *scales_fp16)
 {
     if (N < 0 || K <= 0) return -1;
     if (rotate && (K & (K - 1))) return -1;
@@ -262,11 +303,7 @@ int oracle_quantize_weights(const uint16_t *w, int N, int K, int64_t ldw, int ro
     for (int n = 0; n < N; ++n) {
         float *v = (float *)malloc(sizeof(float) * (size_t)K);
         if (!v) { err = 1; continue; }
-        for (int k = 0; k < K; ++k) v[k] = half_bits_to_float(w[(int64_t)n * ldw + k]);
-        if (rotate) {
-            oracle_fwht_f32(v, K);
-            for (int k = 0; k < K; ++k) v[k] = v[k] * norm;
-        }
+        act_row(w + (int64_t)n * ldw, K, rotate, ch_mul, norm, v);
         float amax = 0.0f;
         for (int k = 0; k < K; ++k) {
             float a = fabsf(v[k]);

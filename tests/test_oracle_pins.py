@@ -212,6 +212,48 @@ def test_quantizer_row_index_and_stride():
     assert np.array_equal(p3, p4) and np.array_equal(s3, s4)
 
 
+def test_per_tensor_and_channel_multiplier_granularities():
+    """Per-tensor: every row carries numpy's global amax / 7, the error bound holds with that one scale, and a
+    one-row tensor gives the per-token result. Channel multiplier: with powers of two it equals quantizing the
+    pre-multiplied fp16 tensor (the products are exact), all ones changes nothing, and dividing the outlier
+    channels down before quantizing (the factor moved into the weights) lowers the error of the W4A4 product."""
+    x = wl.activations(51, 3, 12, 256, 4, 30.0)
+    for rot in (False, True):
+        packed, s, codes = oracle.quantize_act(bits(x), rotate=rot, per_tensor=True)
+        v = oracle.rotate_rows(bits(x), rotate=rot)
+        g = np.abs(v).max()
+        assert (s == np.float32(g) / np.float32(7.0)).all()
+        assert (np.abs(v.astype(np.float64) - s[:, None].astype(np.float64) * codes) <= s[0] / 2 * (1 + 2.0 ** -20)).all()
+        assert np.array_equal(oracle.unpack_nibbles(packed), codes)
+        p1, s1, c1 = oracle.quantize_act(bits(x[3:4]), rotate=rot, per_tensor=True)
+        p0, s0, c0 = oracle.quantize_act(bits(x[3:4]), rotate=rot)
+        assert np.array_equal(c1, c0) and np.array_equal(s1, s0)
+    m = np.exp2(np.arange(256) % 5 - 2).astype(np.float32)                       # 1/4 .. 4
+    pre = (x.astype(np.float32) * m).astype(np.float16)
+    assert np.array_equal(pre.astype(np.float32), x.astype(np.float32) * m)      # exact in fp16
+    for rot in (False, True):
+        a = oracle.quantize_act(bits(x), rotate=rot, ch_mul=m)
+        b = oracle.quantize_act(bits(pre), rotate=rot)
+        assert np.array_equal(a[2], b[2]) and np.array_equal(a[1], b[1])
+        c = oracle.quantize_act(bits(x), rotate=rot, ch_mul=np.ones(256, np.float32))
+        d = oracle.quantize_act(bits(x), rotate=rot)
+        assert np.array_equal(c[0], d[0]) and np.array_equal(c[1], d[1])
+    # smoothing: divide each channel by its typical magnitude, multiply the weights' columns by it
+    N, K, M = 32, 256, 12
+    w = _fp16_weights(52, N, K)
+    ref = x.astype(np.float64) @ w.astype(np.float64).T
+    d = np.maximum(np.abs(x.astype(np.float32)).max(axis=0), np.float32(1e-3))
+    d = np.exp2(np.round(0.5 * np.log2(d))).astype(np.float32)                   # half the outlier scale moves into the
+                                                                                 # weights; powers of two: 1/d exact
+    errs = []
+    for mul_x, mul_w in ((None, None), (1.0 / d, d)):
+        wc, ws = oracle.quantize_weights(bits(w), ch_mul=mul_w)
+        _, sx, xc = oracle.quantize_act(bits(x), ch_mul=None if mul_x is None else mul_x.astype(np.float32))
+        y = oracle.gemm_i32(xc, wc).astype(np.float64) * sx[:, None] * ws.view(np.float16).astype(np.float64)[None, :]
+        errs.append(np.sqrt(np.mean((y - ref) ** 2)) / np.sqrt(np.mean(ref ** 2)))
+    assert errs[1] < 0.7 * errs[0], errs
+
+
 # ------------------------------------------------------------------ offline weight quantizer
 
 def _fp16_weights(seed, N, K, outlier_cols=0):
