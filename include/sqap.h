@@ -47,6 +47,7 @@ typedef enum {
 
 /* Flags of sqap_quantize_act. */
 #define SQAP_Q_ROTATE 1u /* apply the orthonormal Hadamard rotation to each row first (Eq. 6) */
+#define SQAP_Q_PER_TENSOR 2u /* sqap_quantize_act_ex: one scale for the whole tensor ("tensor-wise quantization") */
 
 /* Flags of sqap_pack_weights. */
 #define SQAP_W_ROTATED 1u /* bookkeeping only: the codes are those of W·H^T (Eq. 6, weight side) */
@@ -83,16 +84,18 @@ sqap_status sqap_pack_weights(const int8_t* codes, const uint16_t* scales_fp16, 
  * Offline weight quantizer ("4-bit weights", per-output-channel symmetric round-to-nearest; with
  * SQAP_Q_ROTATE the weight side of Eq. 6: the codes are those of W H^T, H = Sylvester-Hadamard / sqrt(K),
  * to be multiplied with activations quantized with SQAP_Q_ROTATE). For every output channel n:
- *   v = fp32(W[n])  [rotated: H v] ; amax = max|v|
+ *   v = fp32(W[n])  [channel_mul: v[k] *= channel_mul[k]]  [rotated: H v] ; amax = max|v|
  *   scale = fp16(amax / 7)  (fp16(1) for an all-zero row; the smallest positive fp16 if that underflows)
  *   code  = clamp(round_half_even(v / fp32(scale)), -8, 7)
- * w_fp16: device fp16 [N rows, ldw elements apart]; codes_out: device int8 [N*K]; scales_out_fp16: device [N].
+ * w_fp16: device fp16 [N rows, ldw elements apart]; channel_mul: device fp32 [K] or NULL (the reciprocal of the
+ * activation side's per-channel multiplier, see sqap_quantize_act_ex); codes_out: device int8 [N*K];
+ * scales_out_fp16: device [N].
  * K % 32 == 0, K <= 32768; rotation needs K a power of two >= 64. The outputs are what sqap_pack_weights takes
  * (pass SQAP_W_ROTATED there for rotated weights). Weights whose amax / 7 exceeds the fp16 range give an
  * infinite scale, which sqap_pack_weights rejects (SQAP_ERR_RANGE). Enqueues on `stream`, does not synchronise.
  */
-sqap_status sqap_quantize_weights(const void* w_fp16, int N, int K, int64_t ldw, uint32_t flags, int8_t* codes_out,
-                                  uint16_t* scales_out_fp16, void* stream);
+sqap_status sqap_quantize_weights(const void* w_fp16, int N, int K, int64_t ldw, uint32_t flags, const float* channel_mul,
+                                  int8_t* codes_out, uint16_t* scales_out_fp16, void* stream);
 
 /* Releases a handle (NULL is accepted). Synchronises the device. */
 sqap_status sqap_free_weights(sqap_weights* w);
@@ -118,6 +121,20 @@ sqap_status sqap_unpack_weights(const sqap_weights* w, int8_t* codes_out_host, u
  */
 sqap_status sqap_quantize_act(const void* x, int M, int K, int64_t ldx, const int32_t* row_index, uint32_t flags,
                               uint8_t* q_packed, float* scales, void* stream);
+
+/*
+ * The activation quantizer in the other granularities the paper names (Sections 2.2, 3, 3.3):
+ *   SQAP_Q_PER_TENSOR  "tensor-wise": amax is taken over all M rows; every scales[i] receives the one scale, so
+ *                      sqap_w4a4_linear is used unchanged
+ *   channel_mul != NULL  "channel-wise", read as a static per-input-channel multiplier (device fp32 [K]) applied to
+ *                      fp32(x) before the rotation and the max-abs (smoothing); put its reciprocal into the weights
+ *                      with sqap_quantize_weights
+ * Everything else (arguments, layout, rounding, SQAP_Q_ROTATE) is as in sqap_quantize_act, to which the call
+ * falls through when neither extension is requested. K <= 16384. These two forms run in plain kernels (one CTA per
+ * row, three launches for per-tensor): they are correct, not tuned.
+ */
+sqap_status sqap_quantize_act_ex(const void* x, int M, int K, int64_t ldx, const int32_t* row_index, uint32_t flags,
+                                 const float* channel_mul, uint8_t* q_packed, float* scales, void* stream);
 
 /* Bytes of caller-provided scratch that sqap_w4a4_linear needs for M rows against a K-column
  * weight matrix (independent of N). Always a multiple of 256. */

@@ -16,11 +16,12 @@ SQAP_OK, SQAP_ERR_INVALID, SQAP_ERR_RANGE, SQAP_ERR_ALIGN, SQAP_ERR_UNSUPPORTED,
 SQAP_STATIC_WORKSPACE_BYTES = 4 * 1024 * 1024 + 8192
 SQAP_FP16, SQAP_BF16, SQAP_I32 = 0, 1, 2
 SQAP_Q_ROTATE = 1
+SQAP_Q_PER_TENSOR = 2
 SQAP_W_ROTATED = 1
 SQAP_L_FORCE_SIMT, SQAP_L_FORCE_TCGEN05, SQAP_L_FORCE_GEMV, SQAP_L_REUSE_EXPANDED, SQAP_L_FORCE_TCGEN05_TS, SQAP_L_FORCE_TCGEN05_PAIR = 1, 2, 4, 8, 16, 32
 
 EXPORTS = ("sqap_pack_weights", "sqap_quantize_weights", "sqap_free_weights", "sqap_weights_info", "sqap_unpack_weights",
-           "sqap_quantize_act", "sqap_workspace_bytes", "sqap_w4a4_linear", "sqap_w4a4_linear_static",
+           "sqap_quantize_act", "sqap_quantize_act_ex", "sqap_workspace_bytes", "sqap_w4a4_linear", "sqap_w4a4_linear_static",
            "sqap_quantize_linear", "sqap_quantize_linear_workspace_bytes",
            "sqap_prune_tokens",
            "sqap_project_center", "sqap_device_status", "sqap_last_cuda_error", "sqap_status_string",
@@ -55,7 +56,8 @@ def lib() -> ctypes.CDLL:
     L = ctypes.CDLL(LIB_PATH)
     vp, i32, i64, u32, sz = ctypes.c_void_p, ctypes.c_int, ctypes.c_int64, ctypes.c_uint32, ctypes.c_size_t
     L.sqap_pack_weights.argtypes = [vp, vp, i32, i32, u32, vp, ctypes.POINTER(vp)]
-    L.sqap_quantize_weights.argtypes = [vp, i32, i32, i64, u32, vp, vp, vp]
+    L.sqap_quantize_weights.argtypes = [vp, i32, i32, i64, u32, vp, vp, vp, vp]
+    L.sqap_quantize_act_ex.argtypes = [vp, i32, i32, i64, vp, u32, vp, vp, vp, vp]
     L.sqap_free_weights.argtypes = [vp]
     L.sqap_weights_info.argtypes = [vp, ctypes.POINTER(i32), ctypes.POINTER(i32), ctypes.POINTER(u32)]
     L.sqap_unpack_weights.argtypes = [vp, vp, vp]
@@ -135,10 +137,16 @@ def sqap_pack_weights(codes, scales_fp16, N: int, K: int, flags: int = 0, stream
     return Weights(out.value, N, K)
 
 
-def sqap_quantize_weights(w_fp16, N: int, K: int, ldw: int, flags: int, codes_out, scales_out_fp16, stream=None):
+def sqap_quantize_weights(w_fp16, N: int, K: int, ldw: int, flags: int, channel_mul, codes_out, scales_out_fp16,
+                          stream=None):
     """fp16 weights [N, ldw] (device) -> int8 codes [N, K] and fp16 scales [N] (device), see include/sqap.h."""
-    _check(lib().sqap_quantize_weights(_ptr(w_fp16), N, K, ldw, flags, _ptr(codes_out), _ptr(scales_out_fp16),
-                                       _stream(stream)), "sqap_quantize_weights")
+    _check(lib().sqap_quantize_weights(_ptr(w_fp16), N, K, ldw, flags, _ptr(channel_mul), _ptr(codes_out),
+                                       _ptr(scales_out_fp16), _stream(stream)), "sqap_quantize_weights")
+
+
+def sqap_quantize_act_ex(x, M: int, K: int, ldx: int, row_index, flags: int, channel_mul, q_packed, scales, stream=None):
+    _check(lib().sqap_quantize_act_ex(_ptr(x), M, K, ldx, _ptr(row_index), flags, _ptr(channel_mul), _ptr(q_packed),
+                                      _ptr(scales), _stream(stream)), "sqap_quantize_act_ex")
 
 
 def sqap_free_weights(w: Weights):

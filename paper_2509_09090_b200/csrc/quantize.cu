@@ -508,6 +508,73 @@ __global__ void __launch_bounds__(R4K_THREADS, 2) quantize_rotate4096_kernel(con
     cp_async_wait_all();
 }
 
+// ---------------------------------------------------------------------------------------------
+// The other activation granularities the paper names (one scale per TENSOR; a per-CHANNEL multiplier applied
+// first), any row length, written for clarity rather than speed: one CTA per row, the row in shared memory as
+// fp32, Hadamard stages one after the other. mode 0: per-token; mode 1: only the row's max-abs, left in
+// scales[row]; mode 2: quantize with the max-abs found in scales[row] (the tensor's, after tensor_max_kernel).
+__global__ void __launch_bounds__(256) quantize_rows_general_kernel(const __half* __restrict__ x, int K, int64_t ldx,
+                                                                    const int32_t* __restrict__ row_index,
+                                                                    const float* __restrict__ ch_mul, int rotate,
+                                                                    float norm, int mode, uint8_t* __restrict__ q,
+                                                                    float* __restrict__ scales) {
+    extern __shared__ float row_f[];   // K floats
+    __shared__ float red[32];
+    const int row = blockIdx.x;
+    const int64_t src = row_index ? static_cast<int64_t>(row_index[row]) : static_cast<int64_t>(row);
+    const __half* xr = x + src * ldx;
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        float v = __half2float(xr[k]);
+        if (ch_mul) v = __fmul_rn(v, ch_mul[k]);
+        row_f[k] = v;
+    }
+    __syncthreads();
+    if (rotate) {
+        for (int h = 1; h < K; h <<= 1) {
+            for (int pr = threadIdx.x; pr < K / 2; pr += blockDim.x) {
+                const int j = (pr / h) * 2 * h + (pr % h);
+                const float a = row_f[j], b = row_f[j + h];
+                row_f[j] = __fadd_rn(a, b);
+                row_f[j + h] = __fsub_rn(a, b);
+            }
+            __syncthreads();
+        }
+        for (int k = threadIdx.x; k < K; k += blockDim.x) row_f[k] = __fmul_rn(row_f[k], norm);
+        __syncthreads();
+    }
+    float amax = 0.0f;
+    if (mode == 2) {
+        amax = scales[row];
+        __syncthreads();   // every thread has read it before thread 0 replaces it with the scale
+    } else {
+        for (int k = threadIdx.x; k < K; k += blockDim.x) amax = fmaxf(amax, fabsf(row_f[k]));
+        amax = block_max(amax, red);
+    }
+    if (mode == 1) {
+        if (threadIdx.x == 0) scales[row] = amax;
+        return;
+    }
+    float scale, inv;
+    scale_of(amax, scale, inv);
+    if (threadIdx.x == 0) scales[row] = scale;
+    uint32_t* qr = reinterpret_cast<uint32_t*>(q + static_cast<int64_t>(row) * (K / 2));
+    for (int c = threadIdx.x; c < K / 8; c += blockDim.x) {
+        uint32_t t[8];
+#pragma unroll
+        for (int i = 0; i < 8; ++i) t[i] = __float_as_uint(__fadd_rn(__fmul_rn(row_f[8 * c + i], inv), MAGIC8));
+        qr[c] = nibbles_of(low_bytes(t[0], t[1], t[2], t[3]), low_bytes(t[4], t[5], t[6], t[7]));
+    }
+}
+
+// scales[0 .. M) hold the rows' max-abs: replace every entry by their maximum.
+__global__ void __launch_bounds__(1024) tensor_max_kernel(float* __restrict__ scales, int M) {
+    __shared__ float red[32];
+    float m = 0.0f;
+    for (int i = threadIdx.x; i < M; i += blockDim.x) m = fmaxf(m, scales[i]);
+    m = block_max(m, red);
+    for (int i = threadIdx.x; i < M; i += blockDim.x) scales[i] = m;
+}
+
 static int num_sms() {
     static int n = 0;
     if (!n) {
@@ -585,6 +652,44 @@ sqap_status quantize_expanded(const __half* x, int M, int K, int64_t ldx, const 
 }
 
 }  // namespace sqap
+
+extern "C" sqap_status sqap_quantize_act_ex(const void* x, int M, int K, int64_t ldx, const int32_t* row_index,
+                                            uint32_t flags, const float* channel_mul, uint8_t* q_packed, float* scales,
+                                            void* stream) {
+    using namespace sqap;
+    if (flags & ~(SQAP_Q_ROTATE | SQAP_Q_PER_TENSOR)) return SQAP_ERR_INVALID;
+    if (!(flags & SQAP_Q_PER_TENSOR) && !channel_mul)   // nothing extended asked for: the tuned per-token kernels
+        return sqap_quantize_act(x, M, K, ldx, row_index, flags, q_packed, scales, stream);
+    const sqap_status st = quantize_check_args(x, M, K, ldx, flags & SQAP_Q_ROTATE);
+    if (st != SQAP_OK || M == 0) return st;
+    if (!q_packed || !scales) return SQAP_ERR_INVALID;
+    if (!aligned16(q_packed)) return SQAP_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(scales) & 3u) || (reinterpret_cast<uintptr_t>(channel_mul) & 3u)) return SQAP_ERR_ALIGN;
+    if (K > 16384) return SQAP_ERR_UNSUPPORTED;   // the row is held in shared memory as fp32
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    const size_t smem = sizeof(float) * static_cast<size_t>(K);
+    if (smem > 48 * 1024) {
+        cudaError_t e = cudaFuncSetAttribute(quantize_rows_general_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
+                                             static_cast<int>(smem));
+        if (e != cudaSuccess) {
+            note_cuda_error(e);
+            return SQAP_ERR_CUDA;
+        }
+    }
+    const int rotate = (flags & SQAP_Q_ROTATE) ? 1 : 0;
+    const float norm = static_cast<float>(1.0 / sqrt(static_cast<double>(K)));
+    const __half* xh = static_cast<const __half*>(x);
+    if (flags & SQAP_Q_PER_TENSOR) {
+        quantize_rows_general_kernel<<<M, 256, smem, s>>>(xh, K, ldx, row_index, channel_mul, rotate, norm, 1, q_packed, scales);
+        tensor_max_kernel<<<1, 1024, 0, s>>>(scales, M);
+        quantize_rows_general_kernel<<<M, 256, smem, s>>>(xh, K, ldx, row_index, channel_mul, rotate, norm, 2, q_packed, scales);
+        count_launch(3);
+    } else {
+        quantize_rows_general_kernel<<<M, 256, smem, s>>>(xh, K, ldx, row_index, channel_mul, rotate, norm, 0, q_packed, scales);
+        count_launch();
+    }
+    return check_launch();
+}
 
 extern "C" sqap_status sqap_quantize_act(const void* x, int M, int K, int64_t ldx, const int32_t* row_index,
                                          uint32_t flags, uint8_t* q_packed, float* scales, void* stream) {

@@ -61,13 +61,18 @@ __global__ void unpack_weights_kernel(const uint8_t* __restrict__ packed, int N,
 // Walsh-Hadamard stages h = 1, 2, 4, ... applied one after the other with a barrier between them
 // (every stage output is one fp32 add of two fixed inputs, so the bits do not depend on the thread map).
 __global__ void __launch_bounds__(256) quantize_weight_rows_kernel(const __half* __restrict__ w, int K, int64_t ldw,
-                                                                   int rotate, float norm, int8_t* __restrict__ codes,
+                                                                   const float* __restrict__ ch_mul, int rotate,
+                                                                   float norm, int8_t* __restrict__ codes,
                                                                    __half* __restrict__ scales) {
     extern __shared__ float row[];   // K floats
     __shared__ float red[8];
     const int n = blockIdx.x;
     const __half* wr = w + static_cast<int64_t>(n) * ldw;
-    for (int k = threadIdx.x; k < K; k += blockDim.x) row[k] = __half2float(wr[k]);
+    for (int k = threadIdx.x; k < K; k += blockDim.x) {
+        float v = __half2float(wr[k]);
+        if (ch_mul) v = __fmul_rn(v, ch_mul[k]);
+        row[k] = v;
+    }
     __syncthreads();
     if (rotate) {
         for (int h = 1; h < K; h <<= 1) {
@@ -192,15 +197,17 @@ fail:
     return st;
 }
 
-sqap_status sqap_quantize_weights(const void* w_fp16, int N, int K, int64_t ldw, uint32_t flags, int8_t* codes_out,
-                                  uint16_t* scales_out_fp16, void* stream) {
+sqap_status sqap_quantize_weights(const void* w_fp16, int N, int K, int64_t ldw, uint32_t flags, const float* channel_mul,
+                                  int8_t* codes_out, uint16_t* scales_out_fp16, void* stream) {
     using namespace sqap;
     if (N < 0 || K <= 0 || ldw < K) return SQAP_ERR_INVALID;
     if (flags & ~SQAP_Q_ROTATE) return SQAP_ERR_INVALID;
     if (N == 0) return SQAP_OK;
     if (!w_fp16 || !codes_out || !scales_out_fp16) return SQAP_ERR_INVALID;
     if (K % 32 != 0) return SQAP_ERR_ALIGN;
-    if ((reinterpret_cast<uintptr_t>(w_fp16) & 1u) || (reinterpret_cast<uintptr_t>(scales_out_fp16) & 1u)) return SQAP_ERR_ALIGN;
+    if ((reinterpret_cast<uintptr_t>(w_fp16) & 1u) || (reinterpret_cast<uintptr_t>(scales_out_fp16) & 1u) ||
+        (reinterpret_cast<uintptr_t>(channel_mul) & 3u))
+        return SQAP_ERR_ALIGN;
     const bool rotate = (flags & SQAP_Q_ROTATE) != 0;
     if (rotate && ((K & (K - 1)) != 0 || K < 64)) return SQAP_ERR_UNSUPPORTED;
     if (K > 32768) return SQAP_ERR_UNSUPPORTED;   // the row is held in shared memory as fp32
@@ -215,7 +222,7 @@ sqap_status sqap_quantize_weights(const void* w_fp16, int N, int K, int64_t ldw,
     }
     const float norm = static_cast<float>(1.0 / sqrt(static_cast<double>(K)));
     quantize_weight_rows_kernel<<<N, 256, smem, static_cast<cudaStream_t>(stream)>>>(
-        static_cast<const __half*>(w_fp16), K, ldw, rotate ? 1 : 0, norm, codes_out, reinterpret_cast<__half*>(scales_out_fp16));
+        static_cast<const __half*>(w_fp16), K, ldw, channel_mul, rotate ? 1 : 0, norm, codes_out, reinterpret_cast<__half*>(scales_out_fp16));
     count_launch();
     return check_launch();
 }

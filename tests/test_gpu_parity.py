@@ -179,7 +179,7 @@ def test_weight_quantizer_bit_exact_and_feeds_the_linear(N, K, rotate):
     wd = G.to_dev(w)
     codes = torch.empty(N, K, dtype=torch.int8, device="cuda")
     scales = torch.empty(N, dtype=torch.float16, device="cuda")
-    B.sqap_quantize_weights(wd, N, K, K, B.SQAP_Q_ROTATE if rotate else 0, codes, scales)
+    B.sqap_quantize_weights(wd, N, K, K, B.SQAP_Q_ROTATE if rotate else 0, None, codes, scales)
     torch.cuda.synchronize()
     co, so = oracle.quantize_weights(bits(w), rotate=rotate)
     assert np.array_equal(codes.cpu().numpy(), co)
@@ -197,18 +197,60 @@ def test_weight_quantizer_bit_exact_and_feeds_the_linear(N, K, rotate):
         handle.close()
 
 
+@pytest.mark.parametrize("M,K,rotate", [(12, 256, False), (12, 256, True), (37, 4096, True), (5, 11008, False),
+                                        (300, 512, True)])
+def test_quantizer_per_tensor_and_channel_multiplier(M, K, rotate):
+    """sqap_quantize_act_ex in its two extra granularities (and both at once) against the oracle, with a row index
+    list; then a smoothed linear end to end: activations times 1/d, weights times d, codes through the GEMM."""
+    x = wl.activations(61, K + M, M + 3, K, max(1, K // 100), 30.0)
+    x[1] = 0
+    idx = [(5 * i + 2) % (M + 3) for i in range(M)]
+    mul = np.exp2((np.arange(K) % 7) - 3).astype(np.float32) * np.float32(1.25)
+    xd, md, ri = G.to_dev(x), G.to_dev(mul), G.to_dev(np.asarray(idx, np.int32))
+    for per_tensor, use_mul in ((True, False), (False, True), (True, True)):
+        q = torch.full((M, K // 2), 0x5A, dtype=torch.uint8, device="cuda")
+        s = torch.full((M,), -1.0, dtype=torch.float32, device="cuda")
+        fl = (B.SQAP_Q_ROTATE if rotate else 0) | (B.SQAP_Q_PER_TENSOR if per_tensor else 0)
+        B.sqap_quantize_act_ex(xd, M, K, K, ri, fl, md if use_mul else None, q, s)
+        torch.cuda.synchronize()
+        po, so, _ = oracle.quantize_act(bits(x), rotate=rotate, row_index=idx, per_tensor=per_tensor,
+                                        ch_mul=mul if use_mul else None)
+        assert np.array_equal(q.cpu().numpy(), po), (per_tensor, use_mul)
+        assert np.array_equal(s.cpu().numpy(), so), (per_tensor, use_mul)
+    # smoothed W4A4 linear: x * (1/d) against W * d
+    N = 40
+    w = (wl.activations(62, N + K, N, K, 0, 1.0).astype(np.float32) * np.float32(0.02)).astype(np.float16)
+    d = np.exp2(np.round(0.5 * np.log2(np.maximum(np.abs(x.astype(np.float32)).max(axis=0), 1e-3)))).astype(np.float32)
+    inv_d = (np.float32(1.0) / d).astype(np.float32)
+    codes = torch.empty(N, K, dtype=torch.int8, device="cuda")
+    scales = torch.empty(N, dtype=torch.float16, device="cuda")
+    B.sqap_quantize_weights(G.to_dev(w), N, K, K, B.SQAP_Q_ROTATE if rotate else 0, G.to_dev(d), codes, scales)
+    co, so_w = oracle.quantize_weights(bits(w), rotate=rotate, ch_mul=d)
+    assert np.array_equal(codes.cpu().numpy(), co) and np.array_equal(scales.cpu().numpy().view(np.uint16), so_w)
+    q = torch.empty(M, K // 2, dtype=torch.uint8, device="cuda")
+    s = torch.empty(M, dtype=torch.float32, device="cuda")
+    B.sqap_quantize_act_ex(xd, M, K, K, ri, B.SQAP_Q_ROTATE if rotate else 0, G.to_dev(inv_d), q, s)
+    handle = B.sqap_pack_weights(codes, scales, N, K)
+    torch.cuda.synchronize()
+    _, sx, xc = oracle.quantize_act(bits(x), rotate=rotate, row_index=idx, ch_mul=inv_d)
+    out = G.linear(q.cpu().numpy(), s.cpu().numpy(), handle)
+    ref = oracle.epilogue(oracle.gemm_i32(xc, co), sx, so_w)
+    assert G.within_tolerance(out, ref).all()
+    handle.close()
+
+
 def test_weight_quantizer_rejects_bad_arguments():
     w = torch.zeros(8 * 96, dtype=torch.float16, device="cuda")
     c = torch.zeros(8 * 96, dtype=torch.int8, device="cuda")
     s = torch.zeros(8, dtype=torch.float16, device="cuda")
     L = B.lib()
     st = lambda *a: L.sqap_quantize_weights(*a, None)
-    assert st(w.data_ptr(), -1, 96, 96, 0, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
-    assert st(w.data_ptr(), 8, 96, 64, 0, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
-    assert st(w.data_ptr(), 8, 48, 48, 0, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_ALIGN
-    assert st(w.data_ptr(), 8, 96, 96, B.SQAP_Q_ROTATE, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_UNSUPPORTED
-    assert st(None, 8, 96, 96, 0, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
-    assert st(w.data_ptr(), 0, 96, 96, 0, None, None) == B.SQAP_OK
+    assert st(w.data_ptr(), -1, 96, 96, 0, None, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
+    assert st(w.data_ptr(), 8, 96, 64, 0, None, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
+    assert st(w.data_ptr(), 8, 48, 48, 0, None, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_ALIGN
+    assert st(w.data_ptr(), 8, 96, 96, B.SQAP_Q_ROTATE, None, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_UNSUPPORTED
+    assert st(None, 8, 96, 96, 0, None, c.data_ptr(), s.data_ptr()) == B.SQAP_ERR_INVALID
+    assert st(w.data_ptr(), 0, 96, 96, 0, None, None, None) == B.SQAP_OK
 
 
 # ------------------------------------------------------------------ linear: small and ragged shapes
