@@ -46,6 +46,8 @@ def lib():
         _lib = ctypes.CDLL(_LIB)
         _lib.oracle_hadamard_norm.restype = ctypes.c_float
         _lib.oracle_dot_i32.restype = ctypes.c_int32
+        _lib.oracle_exp2_neg.restype = ctypes.c_float
+        _lib.oracle_exp2_neg.argtypes = [ctypes.c_float]
     return _lib
 
 
@@ -104,6 +106,21 @@ def rotate_rows(x_bits, rotate=True):
     M, K = x.shape
     out = np.empty((M, K), np.float32)
     lib().oracle_rotate_rows(_p(x), M, K, ctypes.c_int64(K), int(rotate), _p(out))
+    return out
+
+
+def exp2_neg(t: float) -> np.float32:
+    return np.float32(lib().oracle_exp2_neg(ctypes.c_float(float(t))))
+
+
+def attention_scores(qkv_bits, batch, rows, query_row, visual_start, n_visual, n_heads, head_dim, q_col0, k_col0):
+    """qkv_bits: uint16 view of fp16 [batch*rows, ldq]. Returns fp16 bits u16 [batch, n_heads, n_visual]."""
+    x = _c(qkv_bits, np.uint16)
+    out = np.empty((batch, n_heads, n_visual), np.uint16)
+    rc = lib().oracle_attention_scores(_p(x), ctypes.c_int64(x.shape[1]), batch, rows, query_row, visual_start, n_visual,
+                                       n_heads, head_dim, q_col0, k_col0, _p(out))
+    if rc != 0:
+        raise ValueError(f"oracle_attention_scores: {rc}")
     return out
 
 

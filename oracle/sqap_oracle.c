@@ -462,6 +462,78 @@ void oracle_project_center(const double Kmat[9], const double Rt[12], const doub
     out_tu_tv[1] = (int32_t)floor(v / patch_h);
 }
 
+/* ---------------------------------------------------------------- attention scores of the query token */
+
+/*
+ * 2^t for t <= 0 in fp32, defined operation by operation so that any implementation gives the same
+ * bits: i = floor(t), f = t - i in [0, 1) (exact), p = the degree-9 Taylor polynomial of 2^f = e^(f ln 2)
+ * in Horner form with separately rounded multiplies and adds, result = p * 2^i (exact). t < -126 gives 0.
+ * Truncation error below 1e-8, so the value is within a few ulp of the true 2^t.
+ */
+static const float EXP2_C[10] = {1.0f, 6.9314718056e-01f, 2.4022650696e-01f, 5.5504108665e-02f, 9.6181291076e-03f,
+                                 1.3333558146e-03f, 1.5403530393e-04f, 1.5252733804e-05f, 1.3215486790e-06f,
+                                 1.0178086009e-07f};
+float oracle_exp2_neg(float t)
+{
+    if (t < -126.0f) return 0.0f;
+    float i = floorf(t);
+    float f = t - i;
+    float p = EXP2_C[9];
+    for (int k = 8; k >= 0; --k) {
+        p = p * f;
+        p = p + EXP2_C[k];
+    }
+    return ldexpf(p, (int)i);
+}
+
+/*
+ * Importance of the visual tokens as seen from one task-query token (Sec. 3.2, strategy 1: "attention
+ * scores ... of a task-query token"), computed from a fused QKV projection output (fp16):
+ * for observation b, head h and visual token j
+ *   l_j  = ( sum_{d} fp32(q[d]) * fp32(k_j[d]) ) * (1/sqrt D)     products and sums fp32, d ascending
+ *   e_j  = 2^((l_j - max_j l) * log2(e))                         oracle_exp2_neg
+ *   a_j  = fp16( e_j / sum_j e_j )                               sum j ascending, fp32 division
+ * (softmax over the visual tokens only). q = row query_row of the observation, columns q_col0 + h*D ..;
+ * k_j = row visual_start + j, columns k_col0 + h*D .. . Output A [batch][n_heads][n_visual] fp16: the
+ * "score rows" that oracle_prune_tokens sums per token.
+ */
+int oracle_attention_scores(const uint16_t *qkv, int64_t ldq, int batch, int rows, int query_row, int visual_start,
+                            int n_visual, int n_heads, int head_dim, int q_col0, int k_col0, uint16_t *scores_fp16)
+{
+    if (batch < 0 || rows <= 0 || query_row < 0 || query_row >= rows || visual_start < 0 || n_visual < 0 ||
+        visual_start + n_visual > rows || n_heads <= 0 || head_dim <= 0)
+        return -1;
+    const float inv_sqrt_d = (float)(1.0 / sqrt((double)head_dim));
+    const float log2e = 1.44269504f;
+    float *l = (float *)malloc(sizeof(float) * (size_t)(n_visual + 1));
+    if (!l) return -2;
+    for (int b = 0; b < batch; ++b)
+        for (int h = 0; h < n_heads; ++h) {
+            const uint16_t *q = qkv + ((int64_t)b * rows + query_row) * ldq + q_col0 + (int64_t)h * head_dim;
+            float m = -INFINITY;
+            for (int j = 0; j < n_visual; ++j) {
+                const uint16_t *k = qkv + ((int64_t)b * rows + visual_start + j) * ldq + k_col0 + (int64_t)h * head_dim;
+                float acc = 0.0f;
+                for (int d = 0; d < head_dim; ++d) {
+                    float prod = half_bits_to_float(q[d]) * half_bits_to_float(k[d]);
+                    acc = acc + prod;
+                }
+                l[j] = acc * inv_sqrt_d;
+                if (l[j] > m) m = l[j];
+            }
+            float sum = 0.0f;
+            for (int j = 0; j < n_visual; ++j) {
+                float t = (l[j] - m) * log2e;
+                l[j] = oracle_exp2_neg(t);
+                sum = sum + l[j];
+            }
+            uint16_t *out = scores_fp16 + ((int64_t)b * n_heads + h) * n_visual;
+            for (int j = 0; j < n_visual; ++j) out[j] = float_to_half_bits(l[j] / sum);
+        }
+    free(l);
+    return 0;
+}
+
 /* a_j = A[0][j] + A[1][j] + ... + A[R-1][j], left to right in fp32 (the per-head rows of
  * attention from the task-query token to the visual tokens, summed). */
 void oracle_score_sum(const uint16_t *A_fp16, int R, int n_visual, float *a)

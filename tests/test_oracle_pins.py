@@ -438,6 +438,48 @@ def test_projection_pinhole_cases():
             assert (gu, gv) == (tu, tv)
 
 
+def test_exp2_polynomial_against_numpy():
+    ts = np.concatenate([-np.linspace(0, 30, 4001), -np.array([0.0, 1.0, 2.0, 0.5, 125.9, 126.0, 127.0, 500.0])]).astype(np.float32)
+    got = np.array([oracle.exp2_neg(t) for t in ts], np.float64)
+    ref = np.exp2(ts.astype(np.float64))
+    ok = ts >= -126
+    assert (np.abs(got[ok] - ref[ok]) <= 4e-7 * ref[ok]).all()
+    assert (got[~ok] == 0).all()
+    assert oracle.exp2_neg(0.0) == 1.0 and oracle.exp2_neg(-1.0) == 0.5 and oracle.exp2_neg(-7.0) == 2.0 ** -7   # exact
+
+
+def test_attention_scores_against_float64_softmax_and_closed_forms():
+    """The query token's attention over the visual tokens: against a float64 softmax(q.k / sqrt D) per head, rows
+    summing to one, uniform keys giving exactly fp16(1/n), and a dominant key taking all the mass."""
+    B_, rows, vs, nv, H, D = 2, 40, 3, 24, 4, 32
+    ld = 3 * H * D
+    rng = np.random.default_rng(5)
+    qkv = (rng.standard_normal((B_ * rows, ld)) * 1.5).astype(np.float16)
+    a = oracle.attention_scores(bits(qkv), B_, rows, rows - 1, vs, nv, H, D, 0, H * D).view(np.float16)
+    x = qkv.astype(np.float64).reshape(B_, rows, ld)
+    for b in range(B_):
+        for h in range(H):
+            q = x[b, rows - 1, h * D:(h + 1) * D]
+            k = x[b, vs:vs + nv, H * D + h * D:H * D + (h + 1) * D]
+            l = k @ q / math.sqrt(D)
+            p = np.exp(l - l.max())
+            p /= p.sum()
+            assert (np.abs(a[b, h].astype(np.float64) - p) <= p * 2.0 ** -10 + 1e-7).all()
+            assert abs(a[b, h].astype(np.float64).sum() - 1.0) < nv * 2.0 ** -11
+    # all keys equal: every e_j = 1, the sum n is exact, a_j = fp16(1/n)
+    qkv2 = qkv.copy().reshape(B_, rows, ld)
+    qkv2[:, vs:vs + nv, H * D:2 * H * D] = qkv2[:, vs:vs + 1, H * D:2 * H * D]
+    a2 = oracle.attention_scores(bits(qkv2.reshape(B_ * rows, ld)), B_, rows, rows - 1, vs, nv, H, D, 0, H * D).view(np.float16)
+    assert (a2 == np.float16(np.float32(1.0) / np.float32(nv))).all()
+    # one key aligned with a large query: it takes everything
+    qkv3 = np.zeros((rows, ld), np.float16)
+    qkv3[rows - 1, :D] = 8.0
+    qkv3[vs + 5, H * D:H * D + D] = 8.0
+    a3 = oracle.attention_scores(bits(qkv3), 1, rows, rows - 1, vs, nv, H, D, 0, H * D).view(np.float16)
+    assert a3[0, 0, 5] == 1.0 and a3[0, 0].astype(np.float32).sum() == 1.0
+    assert (a3[0, 1] == np.float16(np.float32(1.0) / np.float32(nv))).all()        # other heads: all logits zero
+
+
 def test_score_sum_is_left_to_right_fp32():
     rng = np.random.default_rng(8)
     A = f16(rng.uniform(0, 1, (32, 40)))
