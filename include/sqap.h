@@ -245,6 +245,25 @@ sqap_status sqap_prune_tokens(const sqap_prune_params* p, const void* scores, co
                               int32_t* kept_idx, int32_t* n_kept, void* stream);
 
 /*
+ * Attention scores of one task-query token over the visual tokens (strategy 1 of Section "Quantization-aware
+ * Pruning Strategies" scores the visual tokens by the attention of a task-query token), computed from the fp16
+ * output of a fused QKV projection. For observation b, head h and visual token j:
+ *   l_j = ( sum_d fp32(q[d]) * fp32(k_j[d]) ) * fp32(1/sqrt(head_dim))     fp32 products and sums, d ascending
+ *   e_j = 2^((l_j - max_j l_j) * 1.44269504f)     2^t = P(t - floor t) * 2^floor(t), P the degree-9 Taylor polynomial
+ *                                                 of e^(f ln 2) in Horner form, fp32, unfused; 0 for t < -126
+ *   a_j = fp16( e_j / sum_j e_j )                 sum over j ascending, fp32 division
+ * i.e. a softmax over the visual tokens only. q = row query_row of the observation, columns q_col0 + h*head_dim ...;
+ * k_j = row visual_start + j, columns k_col0 + h*head_dim ... . qkv: device fp16 [batch*rows rows, ldq apart].
+ * scores_out: device fp16 [batch][n_heads][n_visual] — exactly the `scores` input of sqap_prune_tokens with
+ * score_rows = n_heads. Every step is an individually rounded fp32 operation in the stated order, so the result is
+ * bit-reproducible. head_dim % 8 == 0, head_dim <= 256, n_visual <= 1024, ldq % 8 == 0, k_col0 % 8 == 0, qkv
+ * 16-byte aligned.
+ */
+sqap_status sqap_attention_scores(const void* qkv, int64_t ldq, int batch, int rows, int query_row, int visual_start,
+                                  int n_visual, int n_heads, int head_dim, int q_col0, int k_col0, void* scores_out,
+                                  void* stream);
+
+/*
  * Host helper (no GPU): robot-aware protection, Eq. 2-3. Projects the world point xyz through the
  * intrinsics Kmat (3x3 row-major) and extrinsics Rt = [R|t] (3x4 row-major) and maps the pixel to
  * token coordinates with the patch size (patch_w, patch_h), in double precision:

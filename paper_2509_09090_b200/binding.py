@@ -23,7 +23,7 @@ SQAP_L_FORCE_SIMT, SQAP_L_FORCE_TCGEN05, SQAP_L_FORCE_GEMV, SQAP_L_REUSE_EXPANDE
 EXPORTS = ("sqap_pack_weights", "sqap_quantize_weights", "sqap_free_weights", "sqap_weights_info", "sqap_unpack_weights",
            "sqap_quantize_act", "sqap_quantize_act_ex", "sqap_workspace_bytes", "sqap_w4a4_linear", "sqap_w4a4_linear_static",
            "sqap_quantize_linear", "sqap_quantize_linear_workspace_bytes",
-           "sqap_prune_tokens",
+           "sqap_prune_tokens", "sqap_attention_scores",
            "sqap_project_center", "sqap_device_status", "sqap_last_cuda_error", "sqap_status_string",
            "sqap_kernel_launch_count")
 
@@ -70,6 +70,7 @@ def lib() -> ctypes.CDLL:
     L.sqap_quantize_linear_workspace_bytes.restype = sz
     L.sqap_quantize_linear.argtypes = [vp, i32, i64, vp, u32, vp, vp, vp, i64, i32, u32, vp, sz, vp]
     L.sqap_prune_tokens.argtypes = [ctypes.POINTER(PruneParams), vp, vp, vp, i64, i32, vp, i64, i32, vp, vp, vp]
+    L.sqap_attention_scores.argtypes = [vp, i64, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp]
     L.sqap_project_center.argtypes = [ctypes.POINTER(ctypes.c_double)] * 3 + [ctypes.c_double, ctypes.c_double,
                                                                               ctypes.POINTER(ctypes.c_int32),
                                                                               ctypes.POINTER(i32)]
@@ -210,6 +211,12 @@ def sqap_prune_tokens(params: dict, scores, ring_center, x, ldx: int, K: int, x_
     _check(lib().sqap_prune_tokens(ctypes.byref(p), _ptr(scores), _ptr(ring_center), _ptr(x), ldx, K, _ptr(x_out),
                                    ldo, out_rows, _ptr(kept_idx), _ptr(n_kept), _stream(stream)),
            "sqap_prune_tokens")
+
+
+def sqap_attention_scores(qkv, ldq: int, batch: int, rows: int, query_row: int, visual_start: int, n_visual: int,
+                          n_heads: int, head_dim: int, q_col0: int, k_col0: int, scores_out, stream=None):
+    _check(lib().sqap_attention_scores(_ptr(qkv), ldq, batch, rows, query_row, visual_start, n_visual, n_heads, head_dim,
+                                       q_col0, k_col0, _ptr(scores_out), _stream(stream)), "sqap_attention_scores")
 
 
 def sqap_project_center(Kmat, Rt, xyz, patch_w: float, patch_h: float):

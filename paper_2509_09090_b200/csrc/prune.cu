@@ -149,7 +149,102 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __half* __restri
     for (int c = threadIdx.x; c < K / 8; c += blockDim.x) d[c] = __ldg(s + c);
 }
 
+// ---------------------------------------------------------------------------------------------
+// Attention of one task-query token to the visual tokens, from a fused QKV projection output: the
+// score rows the criterion above consumes. One CTA per (head, observation); thread = visual token.
+// Every floating-point step is an explicitly rounded fp32 operation in a stated order (sqap.h), so
+// the scores, and with them the kept set, do not depend on this kernel's thread mapping.
+constexpr int ATTN_MAX_HEAD_DIM = 256;
+
+// 2^t for t <= 0: floor / fraction split, degree-9 Taylor polynomial of e^(f ln 2) in Horner form with
+// separately rounded multiplies and adds, exact scaling by 2^floor(t); 0 below -126.
+__device__ __forceinline__ float exp2_neg(float t) {
+    constexpr float c[10] = {1.0f, 6.9314718056e-01f, 2.4022650696e-01f, 5.5504108665e-02f, 9.6181291076e-03f,
+                             1.3333558146e-03f, 1.5403530393e-04f, 1.5252733804e-05f, 1.3215486790e-06f,
+                             1.0178086009e-07f};
+    if (t < -126.0f) return 0.0f;
+    const float i = floorf(t);
+    const float f = __fsub_rn(t, i);
+    float p = c[9];
+#pragma unroll
+    for (int k = 8; k >= 0; --k) p = __fadd_rn(__fmul_rn(p, f), c[k]);
+    return __int_as_float(__float_as_int(p) + (static_cast<int>(i) << 23));   // p in [1, 2], i >= -126: stays normal
+}
+
+__global__ void __launch_bounds__(256) attention_scores_kernel(const __half* __restrict__ qkv, int64_t ldq, int rows,
+                                                               int query_row, int visual_start, int n_visual,
+                                                               int head_dim, int q_col0, int k_col0, float inv_sqrt_d,
+                                                               __half* __restrict__ out) {
+    __shared__ float qf[ATTN_MAX_HEAD_DIM];
+    __shared__ float lg[PRUNE_MAX_VISUAL];
+    __shared__ float red[32];
+    __shared__ float s_sum;
+    const int h = blockIdx.x, b = blockIdx.y, n_heads = gridDim.x;
+    const __half* q = qkv + (static_cast<int64_t>(b) * rows + query_row) * ldq + q_col0 + static_cast<int64_t>(h) * head_dim;
+    for (int d = threadIdx.x; d < head_dim; d += blockDim.x) qf[d] = __half2float(q[d]);
+    __syncthreads();
+    float m = -INFINITY;
+    for (int j = threadIdx.x; j < n_visual; j += blockDim.x) {
+        const __half* k = qkv + (static_cast<int64_t>(b) * rows + visual_start + j) * ldq + k_col0 + static_cast<int64_t>(h) * head_dim;
+        float acc = 0.0f;
+        for (int d = 0; d < head_dim; d += 8) {   // head_dim % 8 == 0: 16-byte loads, sums in d order
+            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(k + d));
+            const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+            for (int i = 0; i < 4; ++i) {
+                const float2 kv = __half22float2(h2[i]);
+                acc = __fadd_rn(acc, __fmul_rn(qf[d + 2 * i], kv.x));
+                acc = __fadd_rn(acc, __fmul_rn(qf[d + 2 * i + 1], kv.y));
+            }
+        }
+        const float l = __fmul_rn(acc, inv_sqrt_d);
+        lg[j] = l;
+        m = fmaxf(m, l);
+    }
+    // block max (exact, order-free)
+#pragma unroll
+    for (int o = 16; o > 0; o >>= 1) m = fmaxf(m, __shfl_xor_sync(0xffffffffu, m, o));
+    if ((threadIdx.x & 31) == 0) red[threadIdx.x >> 5] = m;
+    __syncthreads();
+    m = red[0];
+    for (int i = 1; i < (blockDim.x >> 5); ++i) m = fmaxf(m, red[i]);
+    for (int j = threadIdx.x; j < n_visual; j += blockDim.x) lg[j] = exp2_neg(__fmul_rn(__fsub_rn(lg[j], m), 1.44269504f));
+    __syncthreads();
+    if (threadIdx.x == 0) {   // the sum's order is part of the definition: j ascending
+        float s = 0.0f;
+        for (int j = 0; j < n_visual; ++j) s = __fadd_rn(s, lg[j]);
+        s_sum = s;
+    }
+    __syncthreads();
+    const float s = s_sum;
+    __half* o = out + (static_cast<int64_t>(b) * n_heads + h) * n_visual;
+    for (int j = threadIdx.x; j < n_visual; j += blockDim.x) o[j] = __float2half_rn(__fdiv_rn(lg[j], s));
+}
+
 }  // namespace sqap
+
+extern "C" sqap_status sqap_attention_scores(const void* qkv, int64_t ldq, int batch, int rows, int query_row,
+                                             int visual_start, int n_visual, int n_heads, int head_dim, int q_col0,
+                                             int k_col0, void* scores_out, void* stream) {
+    using namespace sqap;
+    if (batch < 0 || rows <= 0 || query_row < 0 || query_row >= rows || visual_start < 0 || n_visual < 0 ||
+        static_cast<int64_t>(visual_start) + n_visual > rows || n_heads <= 0 || head_dim <= 0 || q_col0 < 0 || k_col0 < 0)
+        return SQAP_ERR_INVALID;
+    if (static_cast<int64_t>(q_col0) + static_cast<int64_t>(n_heads) * head_dim > ldq ||
+        static_cast<int64_t>(k_col0) + static_cast<int64_t>(n_heads) * head_dim > ldq)
+        return SQAP_ERR_INVALID;
+    if (n_visual > PRUNE_MAX_VISUAL || head_dim > ATTN_MAX_HEAD_DIM || batch > 65535) return SQAP_ERR_UNSUPPORTED;
+    if (batch == 0 || n_visual == 0) return SQAP_OK;
+    if (!qkv || !scores_out) return SQAP_ERR_INVALID;
+    if (head_dim % 8 != 0 || ldq % 8 != 0 || k_col0 % 8 != 0 || !aligned16(qkv)) return SQAP_ERR_ALIGN;
+    const float inv_sqrt_d = static_cast<float>(1.0 / sqrt(static_cast<double>(head_dim)));
+    dim3 grid(n_heads, batch);
+    attention_scores_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+        static_cast<const __half*>(qkv), ldq, rows, query_row, visual_start, n_visual, head_dim, q_col0, k_col0, inv_sqrt_d,
+        static_cast<__half*>(scores_out));
+    count_launch();
+    return check_launch();
+}
 
 extern "C" sqap_status sqap_prune_tokens(const sqap_prune_params* p, const void* scores, const int32_t* ring_center,
                                          const void* x, int64_t ldx, int K, void* x_out, int64_t ldo, int out_rows,

@@ -3,6 +3,8 @@
 Bar: INT4 codes, activation scales, int32 accumulators and kept-token indices bit-exact; fp16 /
 bf16 outputs within max(1 ulp, 2e-3 relative) of the oracle's.
 """
+import math
+
 import numpy as np
 import pytest
 
@@ -434,6 +436,30 @@ def test_prune_fps_worked_example():
     p = wl.prune_params(1, 256, 0, 256, 16, 16, 0, 0, 5)
     kept, nk, _ = G.prune(p, np.zeros((1, 256), np.float32))
     assert kept[0, :5].tolist() == [0, 15, 119, 240, 255]
+
+
+@pytest.mark.parametrize("batch,rows,vs,nv,H,D", [(2, 40, 3, 24, 4, 32), (3, 288, 1, 256, 32, 128), (1, 70, 0, 64, 2, 8)])
+def test_attention_scores_bit_exact_and_feed_the_criterion(batch, rows, vs, nv, H, D):
+    """sqap_attention_scores against the oracle (fp16 bits), then scores -> criterion on the device against the
+    oracle's kept rows: quantizer output -> attention -> pruning without leaving the GPU."""
+    ld = 3 * H * D
+    qkv = (wl.activations(71, rows + D, batch * rows, ld, 0, 1.0).astype(np.float32) * np.float32(1.2)).astype(np.float16)
+    qd = G.to_dev(qkv)
+    sc = torch.empty(batch, H, nv, dtype=torch.float16, device="cuda")
+    B.sqap_attention_scores(qd, ld, batch, rows, rows - 1, vs, nv, H, D, 0, H * D, sc)
+    torch.cuda.synchronize()
+    so = oracle.attention_scores(bits(qkv), batch, rows, rows - 1, vs, nv, H, D, 0, H * D)
+    assert np.array_equal(sc.cpu().numpy().view(np.uint16), so)
+    gw = int(round(math.sqrt(nv))) if int(round(math.sqrt(nv))) ** 2 == nv else nv
+    p = wl.prune_params(batch, rows, vs, nv, gw, nv // gw, H, nv // 4, nv // 2, ring_radius=-1)
+    kept = torch.empty(batch, rows, dtype=torch.int32, device="cuda")
+    nk = torch.empty(batch, dtype=torch.int32, device="cuda")
+    B.sqap_prune_tokens(p, sc, None, None, 0, 0, None, 0, 0, kept, nk)
+    torch.cuda.synchronize()
+    ko, no = oracle.prune_tokens(p, so, None)
+    assert np.array_equal(nk.cpu().numpy(), no)
+    for b in range(batch):
+        assert np.array_equal(kept.cpu().numpy()[b, :no[b]], ko[b, :no[b]])
 
 
 def test_prune_rejects_bad_arguments():
