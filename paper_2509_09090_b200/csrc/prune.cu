@@ -72,37 +72,39 @@ __global__ void __launch_bounds__(512) prune_select_kernel(sqap_prune_params p, 
     if (local_union) atomicAdd(&s_union, local_union);
     __syncthreads();
 
-    // Strategy 3 (Eq. 5): farthest-point sampling by one warp. Key = D << 10 | (1023 - j): the
-    // maximum key is the largest distance, lowest index on ties; 0 marks "not a candidate".
+    // Strategy 3 (Eq. 5): farthest-point sampling by one warp. Each candidate keeps ONE word, key = D << 10 |
+    // (1023 - j): the maximum key is the largest distance, lowest index on ties, and since the index bits of a
+    // candidate never change, min over distances is min over keys, so a step is one min per candidate, one warp
+    // max-reduction and no division (the picked token's coordinates come from a reciprocal multiply).
+    // D = 0 marks "picked or never a candidate": such keys lose against every live candidate.
     const int m_fps = max(0, p.keep_total - s_union);
     if (warp == 0 && m_fps > 0) {
-        uint32_t D[CAND];
+        uint32_t key[CAND];
         int tu[CAND], tv[CAND];
+        const uint32_t inv_w = 0xFFFFFFFFu / static_cast<uint32_t>(p.grid_w) + 1u;   // j / grid_w = umulhi(j, inv_w), j < 2^16
 #pragma unroll
         for (int i = 0; i < CAND; ++i) {
             const int j = lane + 32 * i;
             const bool cand = j < nv && keep[j] == 0;
-            D[i] = cand ? FPS_D_INIT : 0u;
-            tu[i] = j % p.grid_w;
+            key[i] = (cand ? (FPS_D_INIT << 10) : 0u) | static_cast<uint32_t>(1023 - (j & 1023));
             tv[i] = j / p.grid_w;
+            tu[i] = j - tv[i] * p.grid_w;
         }
         for (int step = 0; step < m_fps; ++step) {
             uint32_t best = 0;
 #pragma unroll
-            for (int i = 0; i < CAND; ++i) {
-                const uint32_t key = D[i] ? ((D[i] << 10) | static_cast<uint32_t>(1023 - (lane + 32 * i))) : 0u;
-                best = max(best, key);
-            }
+            for (int i = 0; i < CAND; ++i) best = max(best, key[i]);
             best = __reduce_max_sync(0xffffffffu, best);
-            if (best == 0) break;  // remainder exhausted
+            if ((best >> 10) == 0) break;  // remainder exhausted
             const int pj = 1023 - static_cast<int>(best & 1023u);
-            const int pu = pj % p.grid_w, pv = pj / p.grid_w;
+            const int pv = static_cast<int>(__umulhi(static_cast<uint32_t>(pj), inv_w));
+            const int pu = pj - pv * p.grid_w;
             if ((pj & 31) == lane) keep[pj] = 2;
 #pragma unroll
             for (int i = 0; i < CAND; ++i) {
                 const int du = tu[i] - pu, dv = tv[i] - pv;
                 const uint32_t d2 = static_cast<uint32_t>(du * du + dv * dv);  // 0 exactly for the picked token
-                D[i] = min(D[i], d2);
+                key[i] = min(key[i], (d2 << 10) | (key[i] & 1023u));
             }
         }
     }
