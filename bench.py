@@ -254,34 +254,33 @@ def dominant_gemm_roofline(torch, B, path: Path, steps: int, peaks: dict):
     # + 18.9 MB int8 activations + 113.2 MB fp16 output = 157.3 MB; part of the output is still in L2 at the end).
     return dict(bound="tensor", kernel="w4a4_tc_pair_kernel: W4A4 linear GEMM, M=4608 N=12288 K=4096 (int8 MMA on CTA "
                                        "pairs, int32 accumulate in tensor memory)",
-                achieved=achieved, peak=peak, unit="TOP/s", frac=achieved / peak, traffic=118.9e6,
+                achieved=achieved, peak=peak, unit="TOP/s", frac=achieved / peak, traffic=119.3e6,
                 peak_source=f"2 x bf16 burst ({peaks['source']})", ms_per_launch=ms)
 
 
-def cpu_baseline(seconds_budget: float = 20.0):
-    """The oracle, as it stands, on the host cores: a bounded sample of the same step (rows of one
-    observation through layer A's linears plus the pruning criterion of that observation)."""
+def cpu_baseline(seconds_budget: float = 15.0):
+    """The oracle, as it stands, on the host cores: a bounded sample of the same step (whole observations through
+    layer A's four linears plus the pruning criterion of those observations), sized to about seconds_budget."""
     import oracle
     oracle.build()
     wts = wl.config4_weights(seed=4)
-    x = wl.config4_inputs(seed=4, batch=1)
-    rows = 8
-    xs = x["x"][0, :rows]
+    x = wl.config4_inputs(seed=4, batch=N_OBS)
     t0 = time.perf_counter()
-    _oracle_layer(oracle, xs, wts)
-    dt = time.perf_counter() - t0
-    rows = int(max(8, min(wl.ROWS, rows * seconds_budget / max(dt, 1e-3) * 0.8)))
-    xs = x["x"][0, :rows]
-    t0 = time.perf_counter()
-    _oracle_layer(oracle, xs, wts)
-    p = wl.prune_params(1, wl.ROWS, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32, K_ATTN, KEEP,
+    _oracle_layer(oracle, x["x"][0, :16], wts)
+    per_row = (time.perf_counter() - t0) / 16
+    n_obs = int(max(1, min(N_OBS, seconds_budget / max(per_row * wl.ROWS, 1e-3))))
+    rows = n_obs * wl.ROWS
+    xs = x["x"][:n_obs].reshape(rows, wl.HIDDEN)
+    p = wl.prune_params(n_obs, wl.ROWS, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32, K_ATTN, KEEP,
                         ring_radius=RING_RADIUS)
-    oracle.prune_tokens(p, x["scores"].view(np.uint16), x["centers"])
+    t0 = time.perf_counter()
+    _oracle_layer(oracle, xs, wts)
+    oracle.prune_tokens(p, x["scores"][:n_obs].view(np.uint16), x["centers"][:n_obs])
     dt = time.perf_counter() - t0
     ops = layer_ops(rows)
     return dict(value=ops / dt / 1e12, unit="TOPS", cores=oracle.num_threads(), kind="oracle",
-                sample=f"{rows} token rows of one observation through one layer's four W4A4 linears + the pruning "
-                       f"criterion of that observation ({dt:.1f} s)", tokens_per_s=rows / dt)
+                sample=f"{n_obs} observations ({rows} token rows) through one layer's four W4A4 linears + the pruning "
+                       f"criterion of those observations ({dt:.1f} s)", tokens_per_s=rows / dt)
 
 
 def _oracle_layer(oracle, x_f16, wts):
