@@ -596,6 +596,105 @@ def run_detail(args):
                                                   "source": peaks["source"]}}))
 
 
+def run_stack(args):
+    """configs[3]: the 32-layer Llama-2-7B linear stack for one observation: a prefill of 288 token rows (pruned to
+    160 after two layers with the full criterion), then 7 single-token decode steps, all launches replayed from one
+    CUDA graph. Random weights generated on the device (3.2 GB packed; timing does not depend on their values).
+    Prints its own JSON line (not the bench line): times, tokens/s and the weight-streaming fraction of HBM."""
+    import torch
+    from paper_2509_09090_b200 import binding as B
+    t = torch
+    t.cuda.set_device(0)
+    dev = t.device("cuda", 0)
+    peaks = measured_peaks()
+    gen = t.Generator(device=dev)
+    gen.manual_seed(3)
+    H, F, Q = wl.HIDDEN, wl.FFN, wl.QKV
+
+    def rand_w(N, K):
+        codes = t.randint(-8, 8, (N, K), dtype=t.int8, device=dev, generator=gen)
+        scales = ((t.rand(N, device=dev, generator=gen) * 0.015 + 0.005) * (16.0 / np.sqrt(K))).to(t.float16)
+        w = B.sqap_pack_weights(codes, scales, N, K)
+        t.cuda.synchronize()
+        return w
+
+    n_layers = 32
+    layers = [dict(qkv=rand_w(Q, H), o=rand_w(H, H), gate=rand_w(F, H), up=rand_w(F, H), down=rand_w(H, F))
+              for _ in range(n_layers)]
+    inp = wl.config4_inputs(seed=3, batch=1)
+    x = t.from_numpy(inp["x"].reshape(wl.ROWS, H)).to(dev)
+    sc, ce = t.from_numpy(inp["scores"]).to(dev), t.from_numpy(inp["centers"]).to(dev)
+    xdec = t.from_numpy(wl.activations(3, wl.T_X2, 7, H, 41, 30.0)).to(dev)
+    keep = 128
+    rows_kept = 32 + keep
+    x1 = t.empty(rows_kept, H, dtype=t.float16, device=dev)
+    kept = t.empty(1, wl.ROWS, dtype=t.int32, device=dev)
+    nk = t.empty(1, dtype=t.int32, device=dev)
+    p = wl.prune_params(1, wl.ROWS, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32, keep // 2, keep, ring_radius=1)
+    M = wl.ROWS
+    qkv = t.empty(M, Q, dtype=t.float16, device=dev)
+    o = t.empty(M, H, dtype=t.float16, device=dev)
+    h = t.empty(M, F, dtype=t.float16, device=dev)
+    d = t.empty(n_layers, M, H, dtype=t.float16, device=dev)
+    nb = B.sqap_quantize_linear_workspace_bytes(M, Q, F)
+    ws = t.empty(nb, dtype=t.uint8, device=dev)
+
+    def lin(xp, m, ldx, w, w_up, out, rot=False):
+        B.sqap_quantize_linear(xp, m, ldx, None, B.SQAP_Q_ROTATE if rot else 0, w, w_up, out, out.shape[-1], B.SQAP_FP16,
+                               0, ws, nb)
+
+    def layer(xin, m, L, dout):
+        lin(xin.data_ptr(), m, H, L["qkv"], None, qkv, rot=True)
+        lin(qkv.data_ptr() + 2 * 2 * H, m, Q, L["o"], None, o)
+        lin(o.data_ptr(), m, H, L["gate"], L["up"], h)
+        lin(h.data_ptr(), m, F, L["down"], None, dout)
+
+    def prefill():
+        for li in range(n_layers):
+            if li == 2:
+                B.sqap_prune_tokens(p, sc, ce, x, H, H, x1, H, rows_kept, kept, nk)
+            layer(x if li < 2 else x1, M if li < 2 else rows_kept, layers[li], d[li])
+
+    def decode():
+        for step in range(7):
+            for li in range(n_layers):
+                layer(xdec[step:step + 1], 1, layers[li], d[li])
+
+    def timed(fn, reps):
+        fn()
+        t.cuda.synchronize()
+        l0 = B.sqap_kernel_launch_count()
+        g = t.cuda.CUDAGraph()
+        with t.cuda.graph(g):
+            fn()
+        launches = B.sqap_kernel_launch_count() - l0
+        g.replay()
+        t.cuda.synchronize()
+        a, b = t.cuda.Event(enable_timing=True), t.cuda.Event(enable_timing=True)
+        a.record()
+        for _ in range(reps):
+            g.replay()
+        b.record()
+        t.cuda.synchronize()
+        return a.elapsed_time(b) / reps, launches
+
+    ms_pre, l_pre = timed(prefill, max(3, args.steps // 10))
+    ms_dec, l_dec = timed(decode, max(3, args.steps // 10))
+    assert B.sqap_device_status() == B.SQAP_OK
+    wbytes = n_layers * (Q * H + H * H + 2 * F * H + H * F) // 2
+    ops_pre = sum(layer_ops(M if li < 2 else rows_kept) for li in range(n_layers))
+    print(json.dumps({
+        "workload": "configs[3]: 32-layer Llama-2-7B W4A4 linear stack, one observation: prefill of 288 rows (pruned to 160 "
+                    "after two layers), then 7 single-token decode steps; CUDA-graph replay; random device weights",
+        "prefill_ms": ms_pre, "prefill_tops": ops_pre / (ms_pre * 1e-3) / 1e12, "prefill_launches": l_pre,
+        "prefill_weight_stream_gbs": wbytes / (ms_pre * 1e-3) / 1e9,
+        "decode_ms_per_token": ms_dec / 7, "decode_launches": l_dec,
+        "decode_weight_stream_gbs": 7 * wbytes / (ms_dec * 1e-3) / 1e9,
+        "decode_frac_of_hbm": 7 * wbytes / (ms_dec * 1e-3) / 1e9 / peaks["hbm_gbs"],
+        "total_ms": ms_pre + ms_dec, "packed_weight_bytes": wbytes,
+        "peaks": {"hbm_gbs": peaks["hbm_gbs"], "source": peaks["source"]}}))
+
+
 def run_single_kernel(args):
     """Profiling aid: a few launches of one kernel of the path on a small, larger-than-L2 case
     (what `ncu -k ... -c 3` captures). Prints nothing that counts as a bench value."""
@@ -649,10 +748,14 @@ def main():
     ap.add_argument("--no-graph", action="store_true", help="issue the step's launches eagerly instead of replaying a CUDA graph")
     ap.add_argument("--detail", action="store_true",
                     help="time every kernel of the path alone at the workload's shapes (one JSON table, no bench line)")
+    ap.add_argument("--stack", action="store_true",
+                    help="time configs[3] (32-layer stack: prefill + 7 decode tokens for one observation); own JSON line")
     ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "quantize", "prune"],
                     help="profiling aid: launch only this kernel --steps times (no bench line)")
     args = ap.parse_args()
-    if args.detail:
+    if args.stack:
+        run_stack(args)
+    elif args.detail:
         run_detail(args)
     elif args.kernel:
         run_single_kernel(args)
