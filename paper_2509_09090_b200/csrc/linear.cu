@@ -333,7 +333,7 @@ static size_t round256(size_t v) { return (v + 255) / 256 * 256; }
 
 namespace sqap {
 
-enum LinearPath { PATH_SIMT, PATH_TC, PATH_TC_TS, PATH_TC_PAIR, PATH_GEMV };
+enum LinearPath { PATH_SIMT, PATH_TC, PATH_TC_TS, PATH_TC_PAIR, PATH_GEMV, PATH_MMA };
 
 // Argument rules shared by the entry points that run a linear (everything except the activation side).
 static sqap_status check_linear_args(int M, const sqap_weights* w, const sqap_weights* w_up, const void* out,
@@ -387,6 +387,9 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
     } else if (flags & SQAP_L_FORCE_TCGEN05_PAIR) {
         if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
         *path = PATH_TC_PAIR;
+    } else if (flags & SQAP_L_FORCE_MMA) {
+        if (!mma_stream_supports(a)) return SQAP_ERR_UNSUPPORTED;
+        *path = PATH_MMA;
     } else {
         // tensor-memory kernels: CTA pairs once there are enough token tiles to fill them, one CTA per tile below
         // the weight-streaming kernel re-reads the activations per row of M, so beyond two rows it only wins where
@@ -403,6 +406,7 @@ static sqap_status run_gemm(const LinearArgs& a, LinearPath path, cudaStream_t s
     if (path == PATH_TC) return launch_linear_tcgen05(a, s);
     if (path == PATH_TC_TS) return launch_linear_tcgen05_ts(a, s);
     if (path == PATH_TC_PAIR) return launch_linear_tcgen05_pair(a, s);
+    if (path == PATH_MMA) return launch_linear_mma_stream(a, s);
     if (path == PATH_GEMV) {
         const int chunks = a.K / 32;
         // rows up to 4096 codes: activation row in registers; longer rows would not amortise loading it

@@ -46,4 +46,10 @@ sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s);
 // The same on CTA pairs (linear_tc_pair.cu): the large-M kernel. Runs every shape the kernels above run.
 sqap_status launch_linear_tcgen05_pair(const LinearArgs& a, cudaStream_t s);
 
+
+// Register-MMA weight streamer for a handful of tokens (linear_mma.cu): K % 128 == 0 and M <= MMA_STREAM_MAX_M.
+constexpr int MMA_STREAM_MAX_M = 32;
+bool mma_stream_supports(const LinearArgs& a);
+sqap_status launch_linear_mma_stream(const LinearArgs& a, cudaStream_t s);
+
 }  // namespace sqap

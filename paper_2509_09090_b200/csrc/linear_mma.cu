@@ -1,0 +1,164 @@
+// W4A4 linear for a handful of tokens (3 <= M <= 32): the call is bound by the HBM stream of the packed
+// weights (N*K/2 bytes), so the kernel is a weight streamer. Nothing is staged: every lane pulls 16-byte pieces
+// of weight rows straight from global memory into registers, masks the two nibble planes apart (two ANDs per
+// word) and feeds them to register-level int8 MMAs (m16n8k32) against the expanded int8 activations, which stay
+// in L1. The register MMA is here only because dp4a cannot keep 16-32 tokens' worth of arithmetic under the
+// HBM time; the tensor-memory kernels need shared-memory and TMEM pipelines whose fill and drain cost more
+// than this whole call.
+//
+// Work split: a CTA owns 16 weight rows (with SwiGLU: the same 16 rows of the gate and of the up matrix); its
+// eight warps take the 128-code blocks of K round-robin and add their partial sums through shared memory
+// (integer sums: the order cannot change the result).
+//
+// Fragment bookkeeping (g = lane / 4, t = lane % 4). The MMA multiplies A (16 rows x 32 k) by B (32 k x 8
+// columns); a lane supplies A words for rows g and g + 8 at k-slots 4t..4t+3 and 16+4t..16+4t+3 and B words for
+// column g at the same k-slots. Which codes sit in which k-slot is free as long as A and B agree, so lane t takes
+// the 16-byte chunk t of the block's 64 packed bytes: word i of that chunk carries codes 16t+4i..16t+4i+3 in its
+// low nibbles and codes 64+16t+4i.. in its high nibbles, and meets words i of the activation row at byte offsets
+// 16t and 64+16t of the block. Four MMAs per block and token group: (words 0,1 low), (2,3 low), (0,1 high),
+// (2,3 high).
+#include "linear.cuh"
+
+namespace sqap {
+
+namespace {
+
+constexpr int MMA_WARPS = 8;
+
+__device__ __forceinline__ void mma_s8(int (&d)[4], uint32_t a0, uint32_t a1, uint32_t a2, uint32_t a3, uint32_t b0,
+                                       uint32_t b1) {
+    asm volatile("mma.sync.aligned.m16n8k32.row.col.s32.s8.s8.s32 {%0,%1,%2,%3}, {%4,%5,%6,%7}, {%8,%9}, {%0,%1,%2,%3};"
+                 : "+r"(d[0]), "+r"(d[1]), "+r"(d[2]), "+r"(d[3])
+                 : "r"(a0), "r"(a1), "r"(a2), "r"(a3), "r"(b0), "r"(b1));
+}
+
+// Weights are read once: keep them out of L1, which holds the activations.
+__device__ __forceinline__ uint4 ld_stream(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
+
+// One block of 128 codes: rows (wa: g, wb: g + 8) against NG token groups.
+template <int NG>
+__device__ __forceinline__ void block_mma(int (&acc)[NG][4], const uint4& wa, const uint4& wb, const uint4 (&xl)[NG],
+                                          const uint4 (&xh)[NG]) {
+    constexpr uint32_t L = 0x0F0F0F0Fu, H = 0xF0F0F0F0u;
+#pragma unroll
+    for (int j = 0; j < NG; ++j) {
+        mma_s8(acc[j], wa.x & L, wb.x & L, wa.y & L, wb.y & L, xl[j].x, xl[j].y);
+        mma_s8(acc[j], wa.z & L, wb.z & L, wa.w & L, wb.w & L, xl[j].z, xl[j].w);
+        mma_s8(acc[j], wa.x & H, wb.x & H, wa.y & H, wb.y & H, xh[j].x, xh[j].y);
+        mma_s8(acc[j], wa.z & H, wb.z & H, wa.w & H, wb.w & H, xh[j].z, xh[j].w);
+    }
+}
+
+// NG = token groups of 8 (M <= 8 * NG).
+template <int NG, bool SWIGLU>
+__global__ void __launch_bounds__(MMA_WARPS * 32) w4a4_mma_kernel(LinearArgs a) {
+    constexpr int SETS = SWIGLU ? 2 : 1;
+    __shared__ int red[MMA_WARPS][SETS * NG * 4][32];
+    const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
+    const int g = lane >> 2, t = lane & 3;
+    const int n0 = blockIdx.x * 16;
+    const int64_t row_bytes = a.K / 2;
+    // rows past N are clamped for the loads and never stored
+    const int r0 = min(n0 + g, a.N - 1), r1 = min(n0 + g + 8, a.N - 1);
+    const uint4* w0 = reinterpret_cast<const uint4*>(a.w + r0 * row_bytes) + t;
+    const uint4* w1 = reinterpret_cast<const uint4*>(a.w + r1 * row_bytes) + t;
+    const uint4* u0 = SWIGLU ? reinterpret_cast<const uint4*>(a.w_up + r0 * row_bytes) + t : nullptr;
+    const uint4* u1 = SWIGLU ? reinterpret_cast<const uint4*>(a.w_up + r1 * row_bytes) + t : nullptr;
+    const uint4* xp[NG];
+    bool xok[NG];
+#pragma unroll
+    for (int j = 0; j < NG; ++j) {
+        const int m = 8 * j + g;
+        xok[j] = m < a.M;
+        xp[j] = reinterpret_cast<const uint4*>(a.x8 + static_cast<int64_t>(xok[j] ? m : 0) * a.K) + t;
+    }
+    int acc[NG][4], accu[SWIGLU ? NG : 1][4];
+#pragma unroll
+    for (int j = 0; j < NG; ++j)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            acc[j][c] = 0;
+            if (SWIGLU) accu[j][c] = 0;
+        }
+
+    const int blocks = a.K / 128;
+#pragma unroll 2
+    for (int b = warp; b < blocks; b += MMA_WARPS) {
+        const uint4 wa = ld_stream(w0 + 4 * b), wb = ld_stream(w1 + 4 * b);
+        uint4 ua = make_uint4(0, 0, 0, 0), ub = make_uint4(0, 0, 0, 0);
+        if (SWIGLU) {
+            ua = ld_stream(u0 + 4 * b);
+            ub = ld_stream(u1 + 4 * b);
+        }
+        uint4 xl[NG], xh[NG];
+#pragma unroll
+        for (int j = 0; j < NG; ++j) {
+            xl[j] = xh[j] = make_uint4(0, 0, 0, 0);   // tokens past M contribute zeros
+            if (xok[j]) {
+                xl[j] = __ldg(xp[j] + 8 * b);
+                xh[j] = __ldg(xp[j] + 8 * b + 4);
+            }
+        }
+        block_mma<NG>(acc, wa, wb, xl, xh);
+        if constexpr (SWIGLU) block_mma<NG>(accu, ua, ub, xl, xh);
+    }
+
+#pragma unroll
+    for (int j = 0; j < NG; ++j)
+#pragma unroll
+        for (int c = 0; c < 4; ++c) {
+            red[warp][j * 4 + c][lane] = acc[j][c];
+            if (SWIGLU) red[warp][NG * 4 + j * 4 + c][lane] = accu[j][c];
+        }
+    __syncthreads();
+    // accumulator word c of lane (g, t), group j = row g + 8 * (c / 2), token 8 j + 2 t + (c % 2)
+    for (int q = threadIdx.x; q < NG * 4 * 32; q += MMA_WARPS * 32) {
+        const int idx = q >> 5, ln = q & 31;
+        const int j = idx >> 2, c = idx & 3;
+        const int n = n0 + (ln >> 2) + ((c & 2) ? 8 : 0);
+        const int m = 8 * j + 2 * (ln & 3) + (c & 1);
+        int raw = 0, raw_u = 0;
+#pragma unroll
+        for (int w = 0; w < MMA_WARPS; ++w) {
+            raw += red[w][idx][ln];
+            if (SWIGLU) raw_u += red[w][NG * 4 + idx][ln];
+        }
+        if (n < a.N && m < a.M) {
+            const int bs = a.bias_sum[m];
+            const float sx = a.act_scales[m];
+            const int tq = finish_acc(raw, bs);
+            float y = dequant(tq, sx, __half2float(a.w_scales[n]));
+            if (SWIGLU) y = swiglu(y, dequant(finish_acc(raw_u, bs), sx, __half2float(a.w_up_scales[n])));
+            store_out(a.out, static_cast<int64_t>(m) * a.ldo + n, a.out_dtype, y, tq);
+        }
+    }
+}
+
+template <int NG>
+void launch_ng(const LinearArgs& a, cudaStream_t s) {
+    const int grid = (a.N + 15) / 16;
+    if (a.w_up) w4a4_mma_kernel<NG, true><<<grid, MMA_WARPS * 32, 0, s>>>(a);
+    else w4a4_mma_kernel<NG, false><<<grid, MMA_WARPS * 32, 0, s>>>(a);
+}
+
+}  // namespace
+
+bool mma_stream_supports(const LinearArgs& a) {
+    return a.half == 64 && a.K % 128 == 0 && a.K >= 128 && a.M >= 1 && a.M <= MMA_STREAM_MAX_M;
+}
+
+sqap_status launch_linear_mma_stream(const LinearArgs& a, cudaStream_t s) {
+    if (!mma_stream_supports(a)) return SQAP_ERR_UNSUPPORTED;
+    if (a.M <= 8) launch_ng<1>(a, s);
+    else if (a.M <= 16) launch_ng<2>(a, s);
+    else if (a.M <= 24) launch_ng<3>(a, s);
+    else launch_ng<4>(a, s);
+    count_launch();
+    return check_launch();
+}
+
+}  // namespace sqap

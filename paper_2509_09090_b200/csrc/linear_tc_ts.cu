@@ -6,14 +6,19 @@
 // weights from shared memory and write them back as int8 for the MMA to read again. Here the unpacked weights
 // never touch shared memory: the unpack warps go from the packed TMA tile through registers (two ANDs per 8
 // weights, see common.cuh) into tensor memory (tcgen05.st), and the MMA takes its A operand from there.
-// Tensor memory (512 columns): two accumulators of 192 columns (the epilogue overlaps the next tile's main
-// loop) + a ring of two 64-column weight tiles (256 int8 per lane).
+// Tensor memory (512 columns): two accumulators (the epilogue overlaps the next tile's main loop) + a ring of
+// 64-column weight tiles (256 int8 per lane): 2 x 192 + 2 tiles, or 2 x 128 + 4 tiles where the token tile is
+// narrow enough.
+// Few tokens make the call a weight stream, and a stage then lives through TMA latency (~1000 cycles) + unpack +
+// MMA + commit before its slot is free again: the ring depths decide the rate. Both are therefore sized at launch
+// from the token-tile width: as many TMA stages as fit in shared memory (3 at 192 tokens, 8 at 16), four weight
+// tiles in tensor memory when the accumulators leave room.
 // One thread issues every MMA, and a tcgen05.mma, a tcgen05.commit or an mbarrier wait each cost it some 60
 // cycles: a pipeline stage therefore covers 256 codes of K (8 MMAs of 96 cycles) per wait and per commit, and
 // a single barrier per stage ("done") releases both the shared-memory slot and the tensor-memory weight tile.
 //
 // Per CTA (persistent, one per SM), warp roles:
-//   warp 0      TMA producer: per stage two boxes of packed weights (128 rows x 64 B, 64B-swizzled) and two
+//   warp 0      TMA producer (converged warp, one elected lane issues): per stage two boxes of packed weights (128 rows x 64 B, 64B-swizzled) and two
 //               boxes of int8 activations (BN rows x 128 B, 128B-swizzled)
 //   warps 2-5   unpack: thread = one tensor-memory lane = one weight row of the tile
 //   warp 1      MMA issuer: 8 x tcgen05.mma (K = 32 each, A in tensor memory) per stage
@@ -31,23 +36,23 @@ constexpr int BM = 128;                   // weight rows per tile (MMA M)
 constexpr int BKH = 128;                  // codes of K per TMA box / per block of the packed weight layout
 constexpr int BK = 2 * BKH;               // codes of K per pipeline stage
 constexpr int BN_MAX = 192;               // tokens per tile (MMA N), runtime BN <= BN_MAX, multiple of 16
-constexpr int S = 3;                      // TMA ring: packed weights + activation tile
-constexpr int U = 2;                      // ring of unpacked weight tiles in tensor memory
-constexpr int XH_BYTES = BN_MAX * BKH;    // 24 KB: one 128-code half of a stage's activation tile
+constexpr int S_MAX = 8;                  // TMA ring (packed weights + activation tile): depth chosen at launch
+constexpr int U_MAX = 4;                  // ring of unpacked weight tiles in tensor memory: 2 or 4
 constexpr int WPH_BYTES = BM * BKH / 2;   // 8 KB: one half of a stage's packed weights
-constexpr int OFF_X = 0;
-constexpr int OFF_WP = OFF_X + S * 2 * XH_BYTES;
-constexpr int OFF_BAR = OFF_WP + S * 2 * WPH_BYTES;
+constexpr int RING_BYTES = 222 * 1024;    // stage s: [weights half 0][weights half 1][tokens half 0][tokens half 1]
+constexpr int OFF_BAR = RING_BYTES;
 constexpr int OFF_TOK = OFF_BAR + 512;    // per-token epilogue constants, two tiles x BN_MAX x 8 bytes
 constexpr int SMEM_BYTES = OFF_TOK + 2 * BN_MAX * 8 + 1024;  // + slack for 1024-byte alignment
-constexpr int TMEM_A_COL = 2 * BN_MAX;    // columns [0,192) and [192,384): accumulators; from 384: weight tiles
 constexpr int A_COLS = BK / 4;            // 64 columns hold 256 int8 per lane
+constexpr int ACC_NARROW = 128;           // accumulator stride (columns) with four weight tiles, else BN_MAX
 constexpr int EPI_WARPS = 8;
 constexpr int THREADS = 32 * (6 + EPI_WARPS);
-static_assert(XH_BYTES % 1024 == 0 && OFF_WP % 1024 == 0, "operand tiles must be 1024-byte aligned");
-static_assert(TMEM_A_COL + U * A_COLS <= 512, "tensor memory budget");
+static_assert(2 * BN_MAX + 2 * A_COLS <= 512 && 2 * ACC_NARROW + U_MAX * A_COLS <= 512, "tensor memory budget");
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
-static_assert(S > U, "a stage's done barrier must not wrap before the unpack warps have seen it");
+static_assert(8 * (3 * S_MAX + U_MAX + 4) + 16 <= 512, "barrier block");
+
+// Bytes of one stage for a token tile of BN rows (BN a multiple of 16: every operand tile stays 1024-byte aligned).
+inline __host__ __device__ int stage_bytes_for(int BN) { return 2 * (WPH_BYTES + BN * BKH); }
 
 // D (tensor memory) += A (tensor memory: lane = row, 4 int8 per 32-bit column) * B (shared memory descriptor).
 // Issued by the lane(s) with issue != 0 of a converged warp.
@@ -81,20 +86,27 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
     const uint32_t base = (smem_u32(smem_raw) + 1023u) & ~1023u;
     uint8_t* sm = smem_raw + (base - smem_u32(smem_raw));
     const uint32_t bar0 = base + OFF_BAR;
-    auto full = [&](int s) { return bar0 + 8u * s; };                  // TMA landed (weights + activations)
-    auto done = [&](int s) { return bar0 + 8u * (S + s); };            // the MMAs of the stage in slot s are done
-    auto wp_empty = [&](int s) { return bar0 + 8u * (2 * S + s); };    // unpack warps have read the packed weights
-    auto a_full = [&](int j) { return bar0 + 8u * (3 * S + j); };      // weight tile j is in tensor memory
-    auto acc_full = [&](int b) { return bar0 + 8u * (3 * S + U + b); };
-    auto acc_empty = [&](int b) { return bar0 + 8u * (3 * S + U + 2 + b); };
-    constexpr int NBAR = 3 * S + U + 4;
+    auto full = [&](int s) { return bar0 + 8u * s; };                      // TMA landed (weights + activations)
+    auto done = [&](int s) { return bar0 + 8u * (S_MAX + s); };            // the MMAs of the stage in slot s are done
+    auto wp_empty = [&](int s) { return bar0 + 8u * (2 * S_MAX + s); };    // unpack warps have read the packed weights
+    auto a_full = [&](int j) { return bar0 + 8u * (3 * S_MAX + j); };      // weight tile j is in tensor memory
+    auto acc_full = [&](int b) { return bar0 + 8u * (3 * S_MAX + U_MAX + b); };
+    auto acc_empty = [&](int b) { return bar0 + 8u * (3 * S_MAX + U_MAX + 2 + b); };
+    constexpr int NBAR = 3 * S_MAX + U_MAX + 4;
+    const int S = a.stages, U = a.a_tiles;     // S > U: a stage's done barrier must not wrap before the unpack warps saw it
+    const uint32_t xh_bytes = static_cast<uint32_t>(a.BN * BKH);
+    const uint32_t stage_bytes = static_cast<uint32_t>(stage_bytes_for(a.BN));
+    auto wp_addr = [&](int s, int h) { return base + s * stage_bytes + h * WPH_BYTES; };
+    auto x_addr = [&](int s, int h) { return base + s * stage_bytes + 2 * WPH_BYTES + h * xh_bytes; };
+    const int acc_stride = U == U_MAX ? ACC_NARROW : BN_MAX;               // accumulator b: columns from b * acc_stride
+    const int tmem_a_col = 2 * acc_stride;                                 // weight tiles from here
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + OFF_BAR + 8 * NBAR);
     volatile int* abort_flag = reinterpret_cast<volatile int*>(sm + OFF_BAR + 8 * NBAR + 8);
 
     const int warp = threadIdx.x >> 5, lane = threadIdx.x & 31;
     const int k_steps = (a.K + BK - 1) / BK;   // a last half-stage past K is zero-filled by TMA and adds nothing
     const int total_tiles = a.m_tiles * a.n_tiles;
-    const uint32_t stage_tx = static_cast<uint32_t>(2 * (WPH_BYTES + a.BN * BKH));
+    const uint32_t stage_tx = stage_bytes;
 
     if (threadIdx.x == 0) {
         for (int s = 0; s < S; ++s) {
@@ -124,36 +136,37 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
     bool failed = false;
 
     if (warp == 0) {
-        // ---------------- TMA producer (one lane)
-        if (lane == 0) {
-            uint32_t it = 0;
-            for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x) {
-                const int n0 = (tile % a.n_tiles) * BM, m0 = (tile / a.n_tiles) * a.BN;
-                for (int ks = 0; ks < k_steps; ++ks, ++it) {
-                    const int s = it % S;
-                    const uint32_t ph = (it / S) & 1u;
-                    if (!mbar_wait(done(s), ph ^ 1u, abort_flag) || !mbar_wait(wp_empty(s), ph ^ 1u, abort_flag)) { failed = true; break; }
-                    mbar_expect_tx(full(s), stage_tx);
+        // ---------------- TMA producer: the whole warp walks the loop, one elected lane issues
+        const uint32_t issue = elect_one();
+        uint32_t it = 0;
+        int s = 0;
+        uint32_t ph = 0;
+        for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x) {
+            const int n0 = (tile % a.n_tiles) * BM, m0 = (tile / a.n_tiles) * a.BN;
+            for (int ks = 0; ks < k_steps; ++ks, ++it) {
+                const bool ok = mbar_wait(done(s), ph ^ 1u, abort_flag) && mbar_wait(wp_empty(s), ph ^ 1u, abort_flag);
+                if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                mbar_expect_tx_if(full(s), stage_tx, issue);
 #pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const uint32_t wp = base + OFF_WP + (2 * s + h) * WPH_BYTES;
-                        const int kc = ks * BK + h * BKH;   // first code of this half
-                        if (a.swiglu) {
-                            tma_load_2d(wp, &tm_w, kc / 2, n0 / 2, full(s));
-                            tma_load_2d(wp + WPH_BYTES / 2, &tm_w_up, kc / 2, n0 / 2, full(s));
-                        } else {
-                            tma_load_2d(wp, &tm_w, kc / 2, n0, full(s));
-                        }
-                        tma_load_2d(base + OFF_X + (2 * s + h) * XH_BYTES, &tm_x, kc, m0, full(s));
+                for (int h = 0; h < 2; ++h) {
+                    const uint32_t wp = wp_addr(s, h);
+                    const int kc = ks * BK + h * BKH;   // first code of this half
+                    if (a.swiglu) {
+                        tma_load_2d_if(wp, &tm_w, kc / 2, n0 / 2, full(s), issue);
+                        tma_load_2d_if(wp + WPH_BYTES / 2, &tm_w_up, kc / 2, n0 / 2, full(s), issue);
+                    } else {
+                        tma_load_2d_if(wp, &tm_w, kc / 2, n0, full(s), issue);
                     }
+                    tma_load_2d_if(x_addr(s, h), &tm_x, kc, m0, full(s), issue);
                 }
+                if (++s == S) { s = 0; ph ^= 1u; }
             }
-            if (failed) {
-                // drain: give every armed stage a bounded chance to land before shared memory is released
-                for (int s = 0; s < S; ++s) {
-                    const uint32_t last = it > static_cast<uint32_t>(s) ? (it - 1 - s) : 0xFFFFFFFFu;
-                    if (last != 0xFFFFFFFFu) mbar_wait(full(last % S), (last / S) & 1u, abort_flag + 1);
-                }
+        }
+        if (failed && issue) {
+            // drain: give every armed stage a bounded chance to land before shared memory is released
+            for (int back = 0; back < S; ++back) {
+                const uint32_t last = it > static_cast<uint32_t>(back) ? (it - 1 - back) : 0xFFFFFFFFu;
+                if (last != 0xFFFFFFFFu) mbar_wait(full(last % S), (last / S) & 1u, abort_flag + 1);
             }
         }
     } else if (warp == 1) {
@@ -162,26 +175,29 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
             const uint32_t issue = elect_one();
             const uint32_t idesc = (2u << 4) | (1u << 7) | (1u << 10) | (static_cast<uint32_t>(a.BN >> 3) << 17) |
                                    (static_cast<uint32_t>(BM >> 4) << 24);
-            uint32_t it = 0, lt = 0;
+            uint32_t lt = 0;
+            int s = 0, j = 0;
+            uint32_t jph = 0;
             for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x, ++lt) {
                 const int b = lt & 1;
                 if (!__all_sync(0xffffffffu, mbar_wait(acc_empty(b), ((lt >> 1) & 1u) ^ 1u, abort_flag))) { failed = true; break; }
                 tc_fence_after();
-                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(b * BN_MAX);
-                for (int ks = 0; ks < k_steps; ++ks, ++it) {
-                    const int s = it % S, j = it % U;
+                const uint32_t d_tmem = tmem_base + static_cast<uint32_t>(b * acc_stride);
+                for (int ks = 0; ks < k_steps; ++ks) {
                     // the unpack warps arrive on a_full(j) only after they saw full(s): this wait covers both operands
-                    if (!__all_sync(0xffffffffu, mbar_wait(a_full(j), (it / U) & 1u, abort_flag))) { failed = true; break; }
+                    if (!__all_sync(0xffffffffu, mbar_wait(a_full(j), jph, abort_flag))) { failed = true; break; }
                     tc_fence_after();
-                    const uint32_t a_tmem = tmem_base + static_cast<uint32_t>(TMEM_A_COL + j * A_COLS);
+                    const uint32_t a_tmem = tmem_base + static_cast<uint32_t>(tmem_a_col + j * A_COLS);
 #pragma unroll
                     for (int h = 0; h < 2; ++h) {
-                        const uint64_t bdesc = smem_desc_sw128(base + OFF_X + (2 * s + h) * XH_BYTES);
+                        const uint64_t bdesc = smem_desc_sw128(x_addr(s, h));
 #pragma unroll
                         for (int k = 0; k < BKH / 32; ++k)
                             tc_mma_i8_ts(d_tmem, a_tmem + 32u * h + 8u * k, bdesc + 2u * k, idesc, (ks | h | k) != 0 ? 1u : 0u, issue);
                     }
                     tc_commit_if(done(s), issue);
+                    if (++s == S) s = 0;
+                    if (++j == U) { j = 0; jph ^= 1u; }
                 }
                 if (failed) break;
                 tc_commit_if(acc_full(b), issue);
@@ -198,17 +214,21 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
         // Consecutive rows then hit different banks for the same c, so the register a chunk lands in is fixed.
         const int sw = (src_row >> 1) & 3;
         uint32_t it = 0;
+        int s = 0, j = 0, sd = 0;      // sd: slot of stage it - U
+        uint32_t ph = 0, phd = 0;
         for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x) {
             for (int ks = 0; ks < k_steps; ++ks, ++it) {
-                const int s = it % S, j = it % U;
-                // weight tile j was last read by the MMAs of stage it - U, whose completion is done((it - U) % S)
-                bool ok = mbar_wait(full(s), (it / S) & 1u, abort_flag);
-                if (ok && it >= U) ok = mbar_wait(done((it - U) % S), ((it - U) / S) & 1u, abort_flag);
+                // weight tile j was last read by the MMAs of stage it - U, whose completion is that stage's done barrier
+                bool ok = mbar_wait(full(s), ph, abort_flag);
+                if (ok && it >= static_cast<uint32_t>(U)) {
+                    ok = mbar_wait(done(sd), phd, abort_flag);
+                    if (++sd == S) { sd = 0; phd ^= 1u; }
+                }
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 tc_fence_after();
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const uint8_t* src = sm + OFF_WP + (2 * s + h) * WPH_BYTES + src_row * 64;
+                    const uint8_t* src = sm + s * stage_bytes + h * WPH_BYTES + src_row * 64;
                     uint32_t r[32];   // column q holds codes k = 4q .. 4q+3 of this half of the row
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
@@ -219,7 +239,7 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
                         r[16 + 4 * c + 2] = v.z & 0xF0F0F0F0u; r[16 + 4 * c + 3] = v.w & 0xF0F0F0F0u;
                     }
                     tc_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
-                                static_cast<uint32_t>(TMEM_A_COL + j * A_COLS + 32 * h), r);
+                                static_cast<uint32_t>(tmem_a_col + j * A_COLS + 32 * h), r);
                 }
                 tc_wait_st();
                 tc_fence_before();
@@ -228,6 +248,8 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
                     mbar_arrive(wp_empty(s));
                     mbar_arrive(a_full(j));
                 }
+                if (++s == S) { s = 0; ph ^= 1u; }
+                if (++j == U) j = 0;
             }
         }
     } else {
@@ -251,7 +273,7 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
             // all epilogue warps leave the loop together if any wait ran out, so the barrier below never hangs
             if (bar_or(1, 32 * EPI_WARPS, !mbar_wait(acc_full(b), (lt >> 1) & 1u, abort_flag))) { failed = true; break; }
             tc_fence_after();
-            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(b * BN_MAX);
+            const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16) + static_cast<uint32_t>(b * acc_stride);
             int n;
             float sw;
             bool n_ok;
@@ -308,6 +330,9 @@ sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s) {
     k.n_tiles = k.swiglu ? (2 * a.N + BM - 1) / BM : (a.N + BM - 1) / BM;
     choose_token_tiles(a.M, k.n_tiles, sm_count(), BN_MAX, 256, &k.m_tiles, &k.BN);
     k.out_dtype = a.out_dtype;
+    k.stages = RING_BYTES / stage_bytes_for(k.BN);
+    if (k.stages > S_MAX) k.stages = S_MAX;
+    k.a_tiles = (k.BN <= ACC_NARROW && k.stages > U_MAX) ? U_MAX : 2;
     k.status = device_status_word();
     if (!k.status) return SQAP_ERR_CUDA;
 

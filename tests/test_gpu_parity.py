@@ -314,6 +314,20 @@ def test_gemv_rows_and_swiglu(M):
     check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_GEMV, B.SQAP_L_FORCE_SIMT, 0])
 
 
+@pytest.mark.parametrize("M,N,K,swiglu", [(1, 16, 128, False), (3, 264, 4096, False), (8, 40, 384, True),
+                                          (9, 130, 1152, False), (16, 1088, 11008, False), (17, 72, 256, True),
+                                          (24, 264, 4096, True), (25, 48, 2048, False), (32, 200, 1024, True)])
+def test_linear_register_mma_streamer(M, N, K, swiglu):
+    """The weight-streaming register-MMA kernel for a handful of tokens: every token-group count (1-4), token
+    counts that leave a group partly empty, channel counts that are not multiples of 16, K blocks that do not
+    divide among the warps evenly, fp16 / bf16 / int32 outputs, with and without the fused gate."""
+    x = wl.activations(28, M + K, M, K, max(1, K // 100), 25.0)
+    g = (wl.weight_codes(28, N + K, N, K), wl.weight_scales(28, N + K, N, mult=0.5))
+    u = (wl.weight_codes(28, N + K + 1, N, K), wl.weight_scales(28, N + K + 1, N, mult=0.5)) if swiglu else None
+    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_MMA, 0])
+    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_MMA], bf16=True)
+
+
 def test_linear_special_operands():
     K = N = 256
     x = wl.activations(22, 1, 16, K, 3, 20.0)
@@ -370,6 +384,12 @@ def test_linear_rejects_bad_arguments():
     assert call(ldo=68) == B.SQAP_ERR_ALIGN
     assert call(wsb=128) == B.SQAP_ERR_NOMEM
     assert call(fl=B.SQAP_L_FORCE_GEMV) == B.SQAP_ERR_UNSUPPORTED
+    # the register-MMA streamer stops at 32 rows (buffers sized for the 40 rows asked for)
+    q40 = torch.zeros(40 * 64, dtype=torch.uint8, device="cuda")
+    s40 = torch.ones(40, dtype=torch.float32, device="cuda")
+    out40 = torch.zeros(40 * 64, dtype=torch.float16, device="cuda")
+    assert L.sqap_w4a4_linear(q40.data_ptr(), s40.data_ptr(), 40, w.handle, None, out40.data_ptr(), 64, B.SQAP_FP16,
+                              B.SQAP_L_FORCE_MMA, ws_t.data_ptr(), 1 << 16, None) == B.SQAP_ERR_UNSUPPORTED
     assert call(fl=3) == B.SQAP_ERR_INVALID
     assert call(M=0) == B.SQAP_OK
     torch.cuda.synchronize()
