@@ -9,17 +9,18 @@
 // Tensor memory (512 columns): two accumulators (the epilogue overlaps the next tile's main loop) + a ring of
 // 64-column weight tiles (256 int8 per lane): 2 x 192 + 2 tiles, or 2 x 128 + 4 tiles where the token tile is
 // narrow enough.
-// Few tokens make the call a weight stream, and a stage then lives through TMA latency (~1000 cycles) + unpack +
-// MMA + commit before its slot is free again: the ring depths decide the rate. Both are therefore sized at launch
-// from the token-tile width: as many TMA stages as fit in shared memory (3 at 192 tokens, 8 at 16), four weight
-// tiles in tensor memory when the accumulators leave room.
+// Both rings are sized at launch from the token-tile width: as many TMA stages as fit in shared memory (3 at 192
+// tokens, 8 at 16), four weight tiles in tensor memory when the accumulators leave room. For narrow tiles this
+// takes TMA latency out of the loop; what remains there is the chain unpack -> MMA -> commit -> unpack, measured
+// at ~750 cycles per stage and CTA however few tokens the tile has (the eight MMAs themselves finish within ~100
+// cycles of their commit), which caps one CTA at 16 KB of weights per ~0.4 us.
 // One thread issues every MMA, and a tcgen05.mma, a tcgen05.commit or an mbarrier wait each cost it some 60
 // cycles: a pipeline stage therefore covers 256 codes of K (8 MMAs of 96 cycles) per wait and per commit, and
 // a single barrier per stage ("done") releases both the shared-memory slot and the tensor-memory weight tile.
 //
 // Per CTA (persistent, one per SM), warp roles:
-//   warp 0      TMA producer (converged warp, one elected lane issues): per stage two boxes of packed weights (128 rows x 64 B, 64B-swizzled) and two
-//               boxes of int8 activations (BN rows x 128 B, 128B-swizzled)
+//   warp 0      TMA producer (converged warp, one elected lane issues): per stage one box of packed weights
+//               (128 rows x 128 B) and two boxes of int8 activations (BN rows x 128 B), all 128B-swizzled
 //   warps 2-5   unpack: thread = one tensor-memory lane = one weight row of the tile
 //   warp 1      MMA issuer: 8 x tcgen05.mma (K = 32 each, A in tensor memory) per stage
 //   warps 6-13  epilogue (as in linear_tc.cu)
@@ -38,8 +39,8 @@ constexpr int BK = 2 * BKH;               // codes of K per pipeline stage
 constexpr int BN_MAX = 192;               // tokens per tile (MMA N), runtime BN <= BN_MAX, multiple of 16
 constexpr int S_MAX = 8;                  // TMA ring (packed weights + activation tile): depth chosen at launch
 constexpr int U_MAX = 4;                  // ring of unpacked weight tiles in tensor memory: 2 or 4
-constexpr int WPH_BYTES = BM * BKH / 2;   // 8 KB: one half of a stage's packed weights
-constexpr int RING_BYTES = 222 * 1024;    // stage s: [weights half 0][weights half 1][tokens half 0][tokens half 1]
+constexpr int W_BYTES = BM * BK / 2;      // 16 KB: a stage's packed weights, 128 rows of 128 bytes
+constexpr int RING_BYTES = 222 * 1024;    // stage s: [weights][tokens half 0][tokens half 1]
 constexpr int OFF_BAR = RING_BYTES;
 constexpr int OFF_TOK = OFF_BAR + 512;    // per-token epilogue constants, two tiles x BN_MAX x 8 bytes
 constexpr int SMEM_BYTES = OFF_TOK + 2 * BN_MAX * 8 + 1024;  // + slack for 1024-byte alignment
@@ -52,7 +53,7 @@ static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 static_assert(8 * (3 * S_MAX + U_MAX + 4) + 16 <= 512, "barrier block");
 
 // Bytes of one stage for a token tile of BN rows (BN a multiple of 16: every operand tile stays 1024-byte aligned).
-inline __host__ __device__ int stage_bytes_for(int BN) { return 2 * (WPH_BYTES + BN * BKH); }
+inline __host__ __device__ int stage_bytes_for(int BN) { return W_BYTES + 2 * BN * BKH; }
 
 // D (tensor memory) += A (tensor memory: lane = row, 4 int8 per 32-bit column) * B (shared memory descriptor).
 // Issued by the lane(s) with issue != 0 of a converged warp.
@@ -96,8 +97,8 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
     const int S = a.stages, U = a.a_tiles;     // S > U: a stage's done barrier must not wrap before the unpack warps saw it
     const uint32_t xh_bytes = static_cast<uint32_t>(a.BN * BKH);
     const uint32_t stage_bytes = static_cast<uint32_t>(stage_bytes_for(a.BN));
-    auto wp_addr = [&](int s, int h) { return base + s * stage_bytes + h * WPH_BYTES; };
-    auto x_addr = [&](int s, int h) { return base + s * stage_bytes + 2 * WPH_BYTES + h * xh_bytes; };
+    auto w_addr = [&](int s) { return base + s * stage_bytes; };
+    auto x_addr = [&](int s, int h) { return base + s * stage_bytes + W_BYTES + h * xh_bytes; };
     const int acc_stride = U == U_MAX ? ACC_NARROW : BN_MAX;               // accumulator b: columns from b * acc_stride
     const int tmem_a_col = 2 * acc_stride;                                 // weight tiles from here
     volatile uint32_t* tmem_slot = reinterpret_cast<volatile uint32_t*>(sm + OFF_BAR + 8 * NBAR);
@@ -147,18 +148,16 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
                 const bool ok = mbar_wait(done(s), ph ^ 1u, abort_flag) && mbar_wait(wp_empty(s), ph ^ 1u, abort_flag);
                 if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
                 mbar_expect_tx_if(full(s), stage_tx, issue);
-#pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint32_t wp = wp_addr(s, h);
-                    const int kc = ks * BK + h * BKH;   // first code of this half
-                    if (a.swiglu) {
-                        tma_load_2d_if(wp, &tm_w, kc / 2, n0 / 2, full(s), issue);
-                        tma_load_2d_if(wp + WPH_BYTES / 2, &tm_w_up, kc / 2, n0 / 2, full(s), issue);
-                    } else {
-                        tma_load_2d_if(wp, &tm_w, kc / 2, n0, full(s), issue);
-                    }
-                    tma_load_2d_if(x_addr(s, h), &tm_x, kc, m0, full(s), issue);
+                // packed weights: rows of 128 bytes (both 128-code blocks of the stage) in one box
+                const uint32_t wp = w_addr(s);
+                if (a.swiglu) {
+                    tma_load_2d_if(wp, &tm_w, ks * (BK / 2), n0 / 2, full(s), issue);
+                    tma_load_2d_if(wp + W_BYTES / 2, &tm_w_up, ks * (BK / 2), n0 / 2, full(s), issue);
+                } else {
+                    tma_load_2d_if(wp, &tm_w, ks * (BK / 2), n0, full(s), issue);
                 }
+#pragma unroll
+                for (int h = 0; h < 2; ++h) tma_load_2d_if(x_addr(s, h), &tm_x, ks * BK + h * BKH, m0, full(s), issue);
                 if (++s == S) { s = 0; ph ^= 1u; }
             }
         }
@@ -210,9 +209,9 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
         // Source row of the packed stage. Plain: row L. SwiGLU: the stage holds 64 gate rows then 64 up rows;
         // within each quadrant lanes 0-15 take gate rows and lanes 16-31 the up rows of the same 16 channels.
         const int src_row = a.swiglu ? (quad * 16 + (lane & 15) + ((lane >> 4) << 6)) : L;
-        // 64-byte rows under the 64B TMA swizzle: 16-byte chunk c of row r sits at chunk c ^ ((r >> 1) & 3).
+        // 128-byte rows under the 128B TMA swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7).
         // Consecutive rows then hit different banks for the same c, so the register a chunk lands in is fixed.
-        const int sw = (src_row >> 1) & 3;
+        const int sw = src_row & 7;
         uint32_t it = 0;
         int s = 0, j = 0, sd = 0;      // sd: slot of stage it - U
         uint32_t ph = 0, phd = 0;
@@ -228,11 +227,11 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
                 tc_fence_after();
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const uint8_t* src = sm + s * stage_bytes + h * WPH_BYTES + src_row * 64;
+                    const uint8_t* src = sm + s * stage_bytes + src_row * 128;
                     uint32_t r[32];   // column q holds codes k = 4q .. 4q+3 of this half of the row
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        const uint4 v = *reinterpret_cast<const uint4*>(src + ((c ^ sw) << 4));
+                        const uint4 v = *reinterpret_cast<const uint4*>(src + (((4 * h + c) ^ sw) << 4));
                         r[4 * c + 0] = v.x & 0x0F0F0F0Fu; r[4 * c + 1] = v.y & 0x0F0F0F0Fu;      // codes 16c .. 16c+15 (+8)
                         r[4 * c + 2] = v.z & 0x0F0F0F0Fu; r[4 * c + 3] = v.w & 0x0F0F0F0Fu;
                         r[16 + 4 * c + 0] = v.x & 0xF0F0F0F0u; r[16 + 4 * c + 1] = v.y & 0xF0F0F0F0u;  // codes 64+16c .. (x16)
@@ -338,8 +337,8 @@ sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s) {
 
     CUtensorMap tm_w, tm_u, tm_x;
     const uint32_t w_box_rows = k.swiglu ? BM / 2 : BM;
-    if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B)) return SQAP_ERR_CUDA;
-    if (!make_map(&tm_u, k.swiglu ? a.w_up : a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B))
+    if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BK / 2, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
+    if (!make_map(&tm_u, k.swiglu ? a.w_up : a.w, a.N, a.K / 2, w_box_rows, BK / 2, CU_TENSOR_MAP_SWIZZLE_128B))
         return SQAP_ERR_CUDA;
     if (!make_map(&tm_x, a.x8, a.M, a.K, k.BN, BKH, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
 

@@ -270,9 +270,11 @@ def test_linear_small_shapes(M, N, K):
 
 @pytest.mark.parametrize("M,N,K,swiglu", [(16, 128, 128, False), (9, 8, 256, False), (257, 130, 384, False),
                                           (144, 320, 1024, False), (700, 200, 512, False), (40, 192, 512, True),
-                                          (300, 64, 256, True), (513, 448, 1152, True), (17, 1088, 11008, False)])
+                                          (300, 64, 256, True), (513, 448, 1152, True), (17, 1088, 11008, False),
+                                          (384, 256, 2304, False), (200, 128, 2048, True)])
 def test_linear_tcgen05_forced(M, N, K, swiglu):
-    """The tensor-core kernel on shapes with ragged token tiles, partial weight tiles and the fused gate."""
+    """The tensor-core kernel on shapes with ragged token tiles, partial weight tiles and the fused gate; the last
+    two walk rings of odd depth (3 and 5 stages) several times around within one tile."""
     x = wl.activations(25, M + K, M, K, max(1, K // 100), 20.0)
     g = (wl.weight_codes(25, N + K, N, K), wl.weight_scales(25, N + K, N, mult=0.5))
     u = (wl.weight_codes(25, N + K + 1, N, K), wl.weight_scales(25, N + K + 1, N, mult=0.5)) if swiglu else None
