@@ -13,9 +13,9 @@
 // Tensor memory per CTA (512 columns): two accumulators of 192 columns + a ring of two 64-column weight tiles.
 //
 // Per CTA, warp roles:
-//   warp 0      TMA producer: per stage two boxes of packed weights (128 rows x 64 B, 64B-swizzled) and two
-//               boxes of int8 activations (BN/2 rows x 128 B, 128B-swizzled); the activation loads of BOTH
-//               CTAs complete on the leader CTA's barrier (the MMA is issued there)
+//   warp 0      TMA producer: per stage one box of packed weights (128 rows x 128 B) and two boxes of int8
+//               activations (BN/2 rows x 128 B), all 128B-swizzled; the activation loads of BOTH CTAs complete
+//               on the leader CTA's barrier (the MMA is issued there)
 //   warps 2-5   unpack: thread = one tensor-memory lane = one weight row of the CTA's tile; signal the leader
 //   warp 1      leader CTA only: 8 x tcgen05.mma.cta_group::2 (M = 256, N = BN, K = 32) per stage
 //   warps 6-13  epilogue of the CTA's own 128 accumulator rows
@@ -182,18 +182,17 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
                     mbar_expect_tx(full(s), w_tx);
                     if (rank == 0) mbar_expect_tx(x_full(s), x_tx);
                     const uint32_t x_bar = map_to_cta(x_full(s), 0);
-#pragma unroll
-                    for (int h = 0; h < 2; ++h) {
-                        const uint32_t wp = base + OFF_WP + (2 * s + h) * WPH_BYTES;
-                        const int kc = ks * BK + h * BKH;   // first code of this half
-                        if (a.swiglu) {
-                            tma_load_2d(wp, &tm_w, kc / 2, n0 / 2, full(s));
-                            tma_load_2d(wp + WPH_BYTES / 2, &tm_w_up, kc / 2, n0 / 2, full(s));
-                        } else {
-                            tma_load_2d(wp, &tm_w, kc / 2, n0, full(s));
-                        }
-                        tma_load_2d_pair(base + OFF_X + (2 * s + h) * XH_BYTES, &tm_x, kc, m0, x_bar);
+                    // packed weights: rows of 128 bytes (both 128-code blocks of the stage) in one box
+                    const uint32_t wp = base + OFF_WP + s * (2 * WPH_BYTES);
+                    if (a.swiglu) {
+                        tma_load_2d(wp, &tm_w, ks * (BK / 2), n0 / 2, full(s));
+                        tma_load_2d(wp + WPH_BYTES, &tm_w_up, ks * (BK / 2), n0 / 2, full(s));
+                    } else {
+                        tma_load_2d(wp, &tm_w, ks * (BK / 2), n0, full(s));
                     }
+#pragma unroll
+                    for (int h = 0; h < 2; ++h)
+                        tma_load_2d_pair(base + OFF_X + (2 * s + h) * XH_BYTES, &tm_x, ks * BK + h * BKH, m0, x_bar);
                 }
             }
             if (failed) {
@@ -245,9 +244,9 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
         // Source row of the packed stage. Plain: row L. SwiGLU: the stage holds 64 gate rows then 64 up rows;
         // within each quadrant lanes 0-15 take gate rows and lanes 16-31 the up rows of the same 16 channels.
         const int src_row = a.swiglu ? (quad * 16 + (lane & 15) + ((lane >> 4) << 6)) : L;
-        // 64-byte rows under the 64B TMA swizzle: 16-byte chunk c of row r sits at chunk c ^ ((r >> 1) & 3).
+        // 128-byte rows under the 128B TMA swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7).
         // Consecutive rows then hit different banks for the same c, so the register a chunk lands in is fixed.
-        const int sw = (src_row >> 1) & 3;
+        const int sw = src_row & 7;
         uint32_t it = 0;
         for (int tile = pair; tile < total_tiles && !failed; tile += n_pairs) {
             for (int ks = 0; ks < k_steps; ++ks, ++it) {
@@ -259,11 +258,11 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
                 tc_fence_after();
 #pragma unroll
                 for (int h = 0; h < 2; ++h) {
-                    const uint8_t* src = sm + OFF_WP + (2 * s + h) * WPH_BYTES + src_row * 64;
+                    const uint8_t* src = sm + OFF_WP + s * (2 * WPH_BYTES) + src_row * 128;
                     uint32_t r[32];   // column q holds codes k = 4q .. 4q+3 of this half of the row
 #pragma unroll
                     for (int c = 0; c < 4; ++c) {
-                        const uint4 v = *reinterpret_cast<const uint4*>(src + ((c ^ sw) << 4));
+                        const uint4 v = *reinterpret_cast<const uint4*>(src + (((4 * h + c) ^ sw) << 4));
                         r[4 * c + 0] = v.x & 0x0F0F0F0Fu; r[4 * c + 1] = v.y & 0x0F0F0F0Fu;      // codes 16c .. 16c+15 (+8)
                         r[4 * c + 2] = v.z & 0x0F0F0F0Fu; r[4 * c + 3] = v.w & 0x0F0F0F0Fu;
                         r[16 + 4 * c + 0] = v.x & 0xF0F0F0F0u; r[16 + 4 * c + 1] = v.y & 0xF0F0F0F0u;  // codes 64+16c .. (x16)
@@ -396,8 +395,8 @@ sqap_status launch_linear_tcgen05_pair(const LinearArgs& a, cudaStream_t s) {
     choose_token_tiles(a.M, k.n_tiles, max_pairs, BN_MAX, 128, &k.m_tiles, &k.BN);
     CUtensorMap tm_w, tm_u, tm_x;
     const uint32_t w_box_rows = k.swiglu ? BM / 2 : BM;
-    if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B)) return SQAP_ERR_CUDA;
-    if (!make_map(&tm_u, k.swiglu ? a.w_up : a.w, a.N, a.K / 2, w_box_rows, BKH / 2, CU_TENSOR_MAP_SWIZZLE_64B))
+    if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BK / 2, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
+    if (!make_map(&tm_u, k.swiglu ? a.w_up : a.w, a.N, a.K / 2, w_box_rows, BK / 2, CU_TENSOR_MAP_SWIZZLE_128B))
         return SQAP_ERR_CUDA;
     if (!make_map(&tm_x, a.x8, a.M, a.K, k.BN / 2, BKH, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
 
