@@ -254,7 +254,7 @@ def dominant_gemm_roofline(torch, B, path: Path, steps: int, peaks: dict):
     # + 18.9 MB int8 activations + 113.2 MB fp16 output = 157.3 MB; part of the output is still in L2 at the end).
     return dict(bound="tensor", kernel="w4a4_tc_pair_kernel: W4A4 linear GEMM, M=4608 N=12288 K=4096 (int8 MMA on CTA "
                                        "pairs, int32 accumulate in tensor memory)",
-                achieved=achieved, peak=peak, unit="TOP/s", frac=achieved / peak, traffic=119.3e6,
+                achieved=achieved, peak=peak, unit="TOP/s", frac=achieved / peak, traffic=118.0e6,
                 peak_source=f"2 x bf16 burst ({peaks['source']})", ms_per_launch=ms)
 
 

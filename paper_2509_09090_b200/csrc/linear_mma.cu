@@ -21,7 +21,7 @@
 
 namespace sqap {
 
-namespace {
+namespace mmas {
 
 constexpr int MMA_WARPS = 8;
 
@@ -145,7 +145,8 @@ void launch_ng(const LinearArgs& a, cudaStream_t s) {
     else w4a4_mma_kernel<NG, false><<<grid, MMA_WARPS * 32, 0, s>>>(a);
 }
 
-}  // namespace
+}  // namespace mmas
+using namespace mmas;
 
 bool mma_stream_supports(const LinearArgs& a) {
     return a.half == 64 && a.K % 128 == 0 && a.K >= 128 && a.M >= 1 && a.M <= MMA_STREAM_MAX_M;
