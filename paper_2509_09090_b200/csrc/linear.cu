@@ -397,8 +397,10 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
         const bool tc_ok = tcgen05_supports(a);
         const int w_tiles = (a.w_up ? 2 * a.N : a.N) / 128;
         // A handful of rows: the register-MMA streamer (its MMA rate holds up to ~16 rows; where the tensor-memory
-        // kernel has too few weight tiles to fill the SMs it stays ahead up to 32). One row: the dp4a streamer.
-        const bool stream = mma_stream_supports(a) && a.M >= 2 && (a.M <= 16 || w_tiles < 64);
+        // kernel has too few weight tiles to fill the SMs it stays ahead up to 32). One row of up to 4096 codes:
+        // the dp4a streamer that keeps the row in registers.
+        const bool one_row_in_registers = a.M == 1 && a.K / 32 <= 32 * 4;   // the dp4a streamer's best case
+        const bool stream = mma_stream_supports(a) && !one_row_in_registers && (a.M <= 16 || w_tiles < 64);
         const bool gemv = !stream && a.M <= 8 && (!tc_ok || a.M <= 2 || (a.M <= 4 && w_tiles < 64));
         *path = stream ? PATH_MMA : gemv ? PATH_GEMV : (tc_ok ? (a.M >= 512 ? PATH_TC_PAIR : PATH_TC_TS) : PATH_SIMT);
     }

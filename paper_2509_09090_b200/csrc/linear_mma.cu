@@ -6,9 +6,9 @@
 // HBM time; the tensor-memory kernels need shared-memory and TMEM pipelines whose fill and drain cost more
 // than this whole call.
 //
-// Work split: a CTA owns 16 weight rows (with SwiGLU: the same 16 rows of the gate and of the up matrix); its
-// eight warps take the 128-code blocks of K round-robin and add their partial sums through shared memory
-// (integer sums: the order cannot change the result).
+// Work split: a row block is 16 weight rows (with SwiGLU: the same 16 rows of the gate and of the up matrix); the
+// eight warps of a CTA take its 128-code blocks of K round-robin and add their partial sums through shared memory
+// (integer sums: the order cannot change the result). CTAs are persistent, two per SM, and walk the row blocks.
 //
 // Fragment bookkeeping (g = lane / 4, t = lane % 4). The MMA multiplies A (16 rows x 32 k) by B (32 k x 8
 // columns); a lane supplies A words for rows g and g + 8 at k-slots 4t..4t+3 and 16+4t..16+4t+3 and B words for
@@ -53,21 +53,30 @@ __device__ __forceinline__ void block_mma(int (&acc)[NG][4], const uint4& wa, co
     }
 }
 
-// NG = token groups of 8 (M <= 8 * NG).
+// A warp's share of one row block is cut into items of KU blocks of 128 codes; the weights of an item are loaded
+// one item ahead of the MMAs that use them (two register buffers), also across row blocks, so that the stream
+// from HBM does not stop while a row block is reduced and written out.
+template <int KU, bool SWIGLU>
+struct ItemWeights {
+    uint4 a[KU], b[KU];                                   // rows g and g + 8
+    uint4 ua[SWIGLU ? KU : 1], ub[SWIGLU ? KU : 1];       // the same rows of the up matrix
+};
+
+// NG = token groups of 8 (M <= 8 * NG). Persistent: CTA c takes row blocks c, c + gridDim.x, ...
 template <int NG, bool SWIGLU>
-__global__ void __launch_bounds__(MMA_WARPS * 32) w4a4_mma_kernel(LinearArgs a) {
+__global__ void __launch_bounds__(MMA_WARPS * 32, 2) w4a4_mma_kernel(LinearArgs a) {
     constexpr int SETS = SWIGLU ? 2 : 1;
+    constexpr int KU = SWIGLU ? (NG <= 2 ? 2 : 1) : (NG <= 2 ? 4 : 2);
     __shared__ int red[MMA_WARPS][SETS * NG * 4][32];
     const int lane = threadIdx.x & 31, warp = threadIdx.x >> 5;
     const int g = lane >> 2, t = lane & 3;
-    const int n0 = blockIdx.x * 16;
     const int64_t row_bytes = a.K / 2;
-    // rows past N are clamped for the loads and never stored
-    const int r0 = min(n0 + g, a.N - 1), r1 = min(n0 + g + 8, a.N - 1);
-    const uint4* w0 = reinterpret_cast<const uint4*>(a.w + r0 * row_bytes) + t;
-    const uint4* w1 = reinterpret_cast<const uint4*>(a.w + r1 * row_bytes) + t;
-    const uint4* u0 = SWIGLU ? reinterpret_cast<const uint4*>(a.w_up + r0 * row_bytes) + t : nullptr;
-    const uint4* u1 = SWIGLU ? reinterpret_cast<const uint4*>(a.w_up + r1 * row_bytes) + t : nullptr;
+    const int blocks = a.K / 128;
+    const int items_per_rb = ((blocks + MMA_WARPS - 1) / MMA_WARPS + KU - 1) / KU;
+    const int n_rb = (a.N + 15) / 16;
+    const int my_rbs = static_cast<int>(blockIdx.x) < n_rb ? (n_rb - 1 - static_cast<int>(blockIdx.x)) / static_cast<int>(gridDim.x) + 1 : 0;
+    const int total_items = my_rbs * items_per_rb;
+
     const uint4* xp[NG];
     bool xok[NG];
 #pragma unroll
@@ -77,70 +86,121 @@ __global__ void __launch_bounds__(MMA_WARPS * 32) w4a4_mma_kernel(LinearArgs a) 
         xp[j] = reinterpret_cast<const uint4*>(a.x8 + static_cast<int64_t>(xok[j] ? m : 0) * a.K) + t;
     }
     int acc[NG][4], accu[SWIGLU ? NG : 1][4];
+    auto clear_acc = [&]() {
 #pragma unroll
-    for (int j = 0; j < NG; ++j)
+        for (int j = 0; j < NG; ++j)
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            acc[j][c] = 0;
-            if (SWIGLU) accu[j][c] = 0;
-        }
+            for (int c = 0; c < 4; ++c) {
+                acc[j][c] = 0;
+                if (SWIGLU) accu[j][c] = 0;
+            }
+    };
+    clear_acc();
 
-    const int blocks = a.K / 128;
-#pragma unroll 2
-    for (int b = warp; b < blocks; b += MMA_WARPS) {
-        const uint4 wa = ld_stream(w0 + 4 * b), wb = ld_stream(w1 + 4 * b);
-        uint4 ua = make_uint4(0, 0, 0, 0), ub = make_uint4(0, 0, 0, 0);
-        if (SWIGLU) {
-            ua = ld_stream(u0 + 4 * b);
-            ub = ld_stream(u1 + 4 * b);
-        }
-        uint4 xl[NG], xh[NG];
+    // block b of item (ci, u): the warps take the blocks of a row round-robin
+    auto block_of = [&](int ci, int u) { return warp + MMA_WARPS * (ci * KU + u); };
+
+    int l_rb = blockIdx.x, l_ci = 0;     // load cursor: row block and item within it
+    auto load_item = [&](ItemWeights<KU, SWIGLU>& w) {
+        const int n0 = l_rb * 16;
+        // rows past N are clamped for the loads and never stored
+        const int64_t o0 = static_cast<int64_t>(min(n0 + g, a.N - 1)) * row_bytes, o1 = static_cast<int64_t>(min(n0 + g + 8, a.N - 1)) * row_bytes;
 #pragma unroll
-        for (int j = 0; j < NG; ++j) {
-            xl[j] = xh[j] = make_uint4(0, 0, 0, 0);   // tokens past M contribute zeros
-            if (xok[j]) {
-                xl[j] = __ldg(xp[j] + 8 * b);
-                xh[j] = __ldg(xp[j] + 8 * b + 4);
+        for (int u = 0; u < KU; ++u) {
+            const int b = block_of(l_ci, u);
+            w.a[u] = w.b[u] = make_uint4(0, 0, 0, 0);
+            if (SWIGLU) w.ua[u] = w.ub[u] = make_uint4(0, 0, 0, 0);
+            if (b < blocks) {
+                w.a[u] = ld_stream(reinterpret_cast<const uint4*>(a.w + o0) + 4 * b + t);
+                w.b[u] = ld_stream(reinterpret_cast<const uint4*>(a.w + o1) + 4 * b + t);
+                if (SWIGLU) {
+                    w.ua[u] = ld_stream(reinterpret_cast<const uint4*>(a.w_up + o0) + 4 * b + t);
+                    w.ub[u] = ld_stream(reinterpret_cast<const uint4*>(a.w_up + o1) + 4 * b + t);
+                }
             }
         }
-        block_mma<NG>(acc, wa, wb, xl, xh);
-        if constexpr (SWIGLU) block_mma<NG>(accu, ua, ub, xl, xh);
-    }
+        if (++l_ci == items_per_rb) { l_ci = 0; l_rb += gridDim.x; }
+    };
 
+    int c_rb = blockIdx.x, c_ci = 0;     // compute cursor
+    auto compute_item = [&](const ItemWeights<KU, SWIGLU>& w) {
 #pragma unroll
-    for (int j = 0; j < NG; ++j)
+        for (int u = 0; u < KU; ++u) {
+            const int b = block_of(c_ci, u);
+            if (b < blocks) {            // uniform over the warp
+                uint4 xl[NG], xh[NG];
 #pragma unroll
-        for (int c = 0; c < 4; ++c) {
-            red[warp][j * 4 + c][lane] = acc[j][c];
-            if (SWIGLU) red[warp][NG * 4 + j * 4 + c][lane] = accu[j][c];
+                for (int j = 0; j < NG; ++j) {
+                    xl[j] = xh[j] = make_uint4(0, 0, 0, 0);   // tokens past M contribute zeros
+                    if (xok[j]) {
+                        xl[j] = __ldg(xp[j] + 8 * b);
+                        xh[j] = __ldg(xp[j] + 8 * b + 4);
+                    }
+                }
+                block_mma<NG>(acc, w.a[u], w.b[u], xl, xh);
+                if constexpr (SWIGLU) block_mma<NG>(accu, w.ua[u], w.ub[u], xl, xh);
+            }
         }
-    __syncthreads();
-    // accumulator word c of lane (g, t), group j = row g + 8 * (c / 2), token 8 j + 2 t + (c % 2)
-    for (int q = threadIdx.x; q < NG * 4 * 32; q += MMA_WARPS * 32) {
-        const int idx = q >> 5, ln = q & 31;
-        const int j = idx >> 2, c = idx & 3;
-        const int n = n0 + (ln >> 2) + ((c & 2) ? 8 : 0);
-        const int m = 8 * j + 2 * (ln & 3) + (c & 1);
-        int raw = 0, raw_u = 0;
+        if (++c_ci < items_per_rb) return;
+        // the row block is complete: add the warps' partial sums (integers: any order) and write it out
+        const int n0 = c_rb * 16;
 #pragma unroll
-        for (int w = 0; w < MMA_WARPS; ++w) {
-            raw += red[w][idx][ln];
-            if (SWIGLU) raw_u += red[w][NG * 4 + idx][ln];
+        for (int j = 0; j < NG; ++j)
+#pragma unroll
+            for (int c = 0; c < 4; ++c) {
+                red[warp][j * 4 + c][lane] = acc[j][c];
+                if (SWIGLU) red[warp][NG * 4 + j * 4 + c][lane] = accu[j][c];
+            }
+        clear_acc();
+        __syncthreads();
+        // accumulator word c of lane (g, t), group j = row g + 8 * (c / 2), token 8 j + 2 t + (c % 2)
+        for (int q = threadIdx.x; q < NG * 4 * 32; q += MMA_WARPS * 32) {
+            const int idx = q >> 5, ln = q & 31;
+            const int j = idx >> 2, c = idx & 3;
+            const int n = n0 + (ln >> 2) + ((c & 2) ? 8 : 0);
+            const int m = 8 * j + 2 * (ln & 3) + (c & 1);
+            int raw = 0, raw_u = 0;
+#pragma unroll
+            for (int w8 = 0; w8 < MMA_WARPS; ++w8) {
+                raw += red[w8][idx][ln];
+                if (SWIGLU) raw_u += red[w8][NG * 4 + idx][ln];
+            }
+            if (n < a.N && m < a.M) {
+                const int bs = a.bias_sum[m];
+                const float sx = a.act_scales[m];
+                const int tq = finish_acc(raw, bs);
+                float y = dequant(tq, sx, __half2float(a.w_scales[n]));
+                if (SWIGLU) y = swiglu(y, dequant(finish_acc(raw_u, bs), sx, __half2float(a.w_up_scales[n])));
+                store_out(a.out, static_cast<int64_t>(m) * a.ldo + n, a.out_dtype, y, tq);
+            }
         }
-        if (n < a.N && m < a.M) {
-            const int bs = a.bias_sum[m];
-            const float sx = a.act_scales[m];
-            const int tq = finish_acc(raw, bs);
-            float y = dequant(tq, sx, __half2float(a.w_scales[n]));
-            if (SWIGLU) y = swiglu(y, dequant(finish_acc(raw_u, bs), sx, __half2float(a.w_up_scales[n])));
-            store_out(a.out, static_cast<int64_t>(m) * a.ldo + n, a.out_dtype, y, tq);
-        }
+        __syncthreads();   // red is free again
+        c_ci = 0;
+        c_rb += gridDim.x;
+    };
+
+    ItemWeights<KU, SWIGLU> w0, w1;
+    if (total_items > 0) load_item(w0);
+    for (int i = 0; i < total_items; i += 2) {
+        if (i + 1 < total_items) load_item(w1);
+        compute_item(w0);
+        if (i + 1 >= total_items) break;
+        if (i + 2 < total_items) load_item(w0);
+        compute_item(w1);
     }
 }
 
 template <int NG>
 void launch_ng(const LinearArgs& a, cudaStream_t s) {
-    const int grid = (a.N + 15) / 16;
+    static int resident = 0;    // CTAs that fit the device at two per SM
+    if (!resident) {
+        int dev = 0, sms = 0;
+        cudaGetDevice(&dev);
+        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
+        resident = 2 * (sms > 0 ? sms : 148);
+    }
+    const int n_rb = (a.N + 15) / 16;
+    const int grid = n_rb < resident ? n_rb : resident;
     if (a.w_up) w4a4_mma_kernel<NG, true><<<grid, MMA_WARPS * 32, 0, s>>>(a);
     else w4a4_mma_kernel<NG, false><<<grid, MMA_WARPS * 32, 0, s>>>(a);
 }
