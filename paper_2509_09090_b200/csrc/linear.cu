@@ -402,7 +402,9 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
         const bool one_row_in_registers = a.M == 1 && a.K / 32 <= 32 * 4;   // the dp4a streamer's best case
         const bool stream = mma_stream_supports(a) && !one_row_in_registers && (a.M <= 16 || w_tiles < 64);
         const bool gemv = !stream && a.M <= 8 && (!tc_ok || a.M <= 2 || (a.M <= 4 && w_tiles < 64));
-        *path = stream ? PATH_MMA : gemv ? PATH_GEMV : (tc_ok ? (a.M >= 512 ? PATH_TC_PAIR : PATH_TC_TS) : PATH_SIMT);
+        // CTA pairs fetch each token once per 256 weight rows: ahead from ~144 tokens on when there are enough pairs
+        const bool pairs = a.M >= 512 || (a.M >= 144 && w_tiles >= 64);
+        *path = stream ? PATH_MMA : gemv ? PATH_GEMV : (tc_ok ? (pairs ? PATH_TC_PAIR : PATH_TC_TS) : PATH_SIMT);
     }
     return SQAP_OK;
 }
