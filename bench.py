@@ -226,7 +226,7 @@ def time_region(torch, fn, steps: int, world: int):
 
 def dominant_gemm_roofline(torch, B, path: Path, steps: int, peaks: dict):
     """The QKV GEMM at M = 4608 (largest single launch), timed alone with CUDA events on its stream.
-    The expand pass is skipped (SQAP_L_REUSE_EXPANDED), so the events bracket exactly one GEMM launch."""
+    The expand pass is skipped (SQAP_L_REUSE_EXPANDED), so the events bracket GEMM launches only."""
     L0, L1 = path.layers
     M, N, K = M_FULL, wl.QKV, wl.HIDDEN
     B.sqap_quantize_act(path.x, M, K, K, None, B.SQAP_Q_ROTATE, path.q, path.sx)
@@ -236,16 +236,12 @@ def dominant_gemm_roofline(torch, B, path: Path, steps: int, peaks: dict):
         B.sqap_w4a4_linear(path.q, path.sx, M, ws[i % 2], None, path.qkv, N, B.SQAP_FP16, B.SQAP_L_REUSE_EXPANDED,
                            path.ws, path.ws_bytes)
     torch.cuda.synchronize()
-    evs = []
-    for i in range(steps):
-        a, b = torch.cuda.Event(enable_timing=True), torch.cuda.Event(enable_timing=True)
-        a.record()
-        B.sqap_w4a4_linear(path.q, path.sx, M, ws[i % 2], None, path.qkv, N, B.SQAP_FP16, B.SQAP_L_REUSE_EXPANDED,
-                           path.ws, path.ws_bytes)
-        b.record()
-        evs.append((a, b))
-    torch.cuda.synchronize()
-    ms = float(np.mean([a.elapsed_time(b) for a, b in evs]))
+    # `reps` launches back to back on one stream (captured once, replayed), CUDA events around the run on that
+    # stream: the average duration of a launch without the host's submission gaps between eager launches
+    reps = max(8, min(steps, 32))
+    ms = graph_time_us(torch, lambda i: B.sqap_w4a4_linear(path.q, path.sx, M, ws[i % 2], None, path.qkv, N, B.SQAP_FP16,
+                                                           B.SQAP_L_REUSE_EXPANDED, path.ws, path.ws_bytes),
+                       reps=reps) * 1e-3
     ops = 2.0 * M * N * K
     achieved = ops / (ms * 1e-3) / 1e12
     peak = 2.0 * peaks["bf16"]       # int8 dense = 2 x bf16 dense (nominal ratio) x the measured bf16 burst figure
@@ -266,8 +262,9 @@ def cpu_baseline(seconds_budget: float = 15.0):
     wts = wl.config4_weights(seed=4)
     x = wl.config4_inputs(seed=4, batch=N_OBS)
     t0 = time.perf_counter()
-    _oracle_layer(oracle, x["x"][0, :16], wts)
-    per_row = (time.perf_counter() - t0) / 16
+    probe = 96    # enough rows to occupy every host thread, as the sample itself does
+    _oracle_layer(oracle, x["x"][0, :probe], wts)
+    per_row = (time.perf_counter() - t0) / probe
     n_obs = int(max(1, min(N_OBS, seconds_budget / max(per_row * wl.ROWS, 1e-3))))
     rows = n_obs * wl.ROWS
     xs = x["x"][:n_obs].reshape(rows, wl.HIDDEN)
@@ -709,12 +706,12 @@ def run_single_kernel(args):
     if args.kernel == "quantize":
         for i in range(args.steps):
             B.sqap_quantize_act(x, M, H, H, None, B.SQAP_Q_ROTATE if i % 2 == 0 else 0, q, sx)
-    elif args.kernel in ("gemm", "gemv", "swiglu"):
-        names = {"gemm": ("qkv",), "gemv": ("qkv",), "swiglu": ("gate", "up")}[args.kernel]
+    elif args.kernel in ("gemm", "gemv", "stream", "swiglu"):
+        names = {"gemm": ("qkv",), "gemv": ("qkv",), "stream": ("qkv",), "swiglu": ("gate", "up")}[args.kernel]
         wts = wl.config4_weights(seed=4)
         ws = [B.sqap_pack_weights(np.ascontiguousarray(wts[n + "_codes"]), np.ascontiguousarray(wts[n + "_scales"]),
                                   wts[n + "_codes"].shape[0], H) for n in names]
-        Mk = 1 if args.kernel == "gemv" else M
+        Mk = {"gemv": 1, "stream": N_OBS}.get(args.kernel, M)   # stream: one decode token per observation
         N = ws[0].N
         out = torch.empty(Mk, N, dtype=torch.float16, device=dev)
         nb = B.sqap_workspace_bytes(Mk, N, H)
@@ -750,7 +747,7 @@ def main():
                     help="time every kernel of the path alone at the workload's shapes (one JSON table, no bench line)")
     ap.add_argument("--stack", action="store_true",
                     help="time configs[3] (32-layer stack: prefill + 7 decode tokens for one observation); own JSON line")
-    ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "quantize", "prune"],
+    ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "stream", "quantize", "prune"],
                     help="profiling aid: launch only this kernel --steps times (no bench line)")
     args = ap.parse_args()
     if args.stack:
