@@ -330,6 +330,19 @@ def test_linear_register_mma_streamer(M, N, K, swiglu):
     check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_MMA], bf16=True)
 
 
+@pytest.mark.parametrize("M,N,K,swiglu", [(1, 136, 4224, False), (16, 8192, 256, False), (17, 8192, 256, False),
+                                          (32, 264, 384, True), (33, 264, 384, True), (143, 8192, 128, False),
+                                          (144, 8192, 128, False), (150, 4096, 256, True)])
+def test_linear_dispatch_boundaries(M, N, K, swiglu):
+    """The kernel the dispatcher picks by itself on either side of each of its thresholds (one row longer than 4096
+    codes; 16 | 17 rows with many weight tiles; 32 | 33 rows with few; 143 | 144 rows with many tiles, plain and
+    gated), against the oracle and against the plain CUDA-core kernel."""
+    x = wl.activations(29, M + K, M, K, max(1, K // 100), 25.0)
+    g = (wl.weight_codes(29, N + K, N, K), wl.weight_scales(29, N + K, N, mult=0.5))
+    u = (wl.weight_codes(29, N + K + 1, N, K), wl.weight_scales(29, N + K + 1, N, mult=0.5)) if swiglu else None
+    check_linear(x, g[0], g[1], up=u, flags_list=[0, B.SQAP_L_FORCE_SIMT])
+
+
 def test_linear_special_operands():
     K = N = 256
     x = wl.activations(22, 1, 16, K, 3, 20.0)
