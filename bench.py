@@ -492,11 +492,20 @@ def kernel_table(torch, B, peaks, device):
     def ncopies(nbytes):
         return max(2, int(np.ceil(L2 / max(nbytes, 1))))
 
+    # what a kernel that does nothing costs as a node of such a graph chain (a one-element torch add): the floor
+    # under every time below; HBM rows shorter than 20 us also get their fraction with the floor taken out
+    tiny = t.zeros(1, device=device)
+    floor_us = graph_time_us(t, lambda i: tiny.add_(1.0), reps=64)
+    rows.append(dict(kernel="empty kernel (graph node floor)", shape="-", bound="latency", us=round(floor_us, 2), note=""))
+
     def add(name, shape, bound, work, us, note=""):
         if bound == "hbm":
             ach = work / (us * 1e-6) / 1e9
-            rows.append(dict(kernel=name, shape=shape, bound="hbm", bytes=work, us=round(us, 2), achieved_gbs=round(ach, 1),
-                             frac=round(ach / hbm, 3), note=note))
+            row = dict(kernel=name, shape=shape, bound="hbm", bytes=work, us=round(us, 2), achieved_gbs=round(ach, 1),
+                       frac=round(ach / hbm, 3), note=note)
+            if us < 20.0 and us > floor_us:
+                row["frac_above_floor"] = round(work / ((us - floor_us) * 1e-6) / 1e9 / hbm, 3)
+            rows.append(row)
         elif bound == "tensor":
             ach = work / (us * 1e-6) / 1e12
             rows.append(dict(kernel=name, shape=shape, bound="tensor", ops=work, us=round(us, 2), achieved_tops=round(ach, 1),

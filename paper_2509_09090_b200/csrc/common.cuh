@@ -20,6 +20,34 @@ int* device_status_word();
 
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
+// Programmatic dependent launch, used along the short kernel chains of a decode step (quantizer -> weight
+// streamer), where a kernel lasts a few microseconds and the gap between two kernels is of the same order.
+// A kernel launched with launch_dependent() may start while the kernel before it in the stream still runs; it does
+// whatever does not depend on that kernel (the streamers: fetch their first weights) and then calls pdl_wait(),
+// which returns once the earlier kernel has completed and its writes are visible. The earlier kernel calls
+// pdl_launch_dependents() as soon as it is running. Both calls do nothing in a kernel launched the plain way.
+constexpr int PDL_MAX_ROWS = 32;   // the quantizers launch this way up to here (the row counts of decode steps)
+#ifdef __CUDACC__
+__device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
+__device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }
+
+template <typename... KArgs, typename... Args>
+inline cudaError_t launch_dependent(void (*kernel)(KArgs...), dim3 grid, dim3 block, size_t smem, cudaStream_t s,
+                                    Args... args) {
+    cudaLaunchConfig_t cfg = {};
+    cfg.gridDim = grid;
+    cfg.blockDim = block;
+    cfg.dynamicSmemBytes = smem;
+    cfg.stream = s;
+    cudaLaunchAttribute attr[1];
+    attr[0].id = cudaLaunchAttributeProgrammaticStreamSerialization;
+    attr[0].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 1;
+    return cudaLaunchKernelEx(&cfg, kernel, static_cast<KArgs>(args)...);
+}
+#endif
+
 // Packed weight matrix in the library's private layout.
 //
 // Codes are stored two per byte, but not as neighbours: the K axis is cut into blocks of

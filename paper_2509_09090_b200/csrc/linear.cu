@@ -245,6 +245,8 @@ __global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
     const int lane = threadIdx.x & 31;
     const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), W = gridDim.x * (blockDim.x >> 5);
     const int chunks = a.K / 32;
+    pdl_launch_dependents();
+    pdl_wait();   // the activation row comes from the kernel before this one
     uint4 xl[CPL], xh[CPL];
 #pragma unroll
     for (int i = 0; i < CPL; ++i) {
@@ -315,8 +317,10 @@ static void launch_gemv1(const LinearArgs& a, cudaStream_t s) {
     }
     const int need = (a.N + 7) / 8;
     const int grid = need < blocks ? need : blocks;
-    if (a.w_up) w4a4_gemv1_kernel<true, CPL><<<grid, 256, 0, s>>>(a);
-    else w4a4_gemv1_kernel<false, CPL><<<grid, 256, 0, s>>>(a);
+    cudaError_t e;
+    if (a.w_up) e = launch_dependent(w4a4_gemv1_kernel<true, CPL>, dim3(grid), dim3(256), 0, s, a);
+    else e = launch_dependent(w4a4_gemv1_kernel<false, CPL>, dim3(grid), dim3(256), 0, s, a);
+    if (e != cudaSuccess) note_cuda_error(e);
 }
 
 template <int MM>

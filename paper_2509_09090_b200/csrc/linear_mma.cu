@@ -181,6 +181,8 @@ __global__ void __launch_bounds__(MMA_WARPS * 32, 2) w4a4_mma_kernel(LinearArgs 
 
     ItemWeights<KU, SWIGLU> w0, w1;
     if (total_items > 0) load_item(w0);
+    pdl_launch_dependents();
+    pdl_wait();   // the activations come from the kernel before this one; the weights above do not
     for (int i = 0; i < total_items; i += 2) {
         if (i + 1 < total_items) load_item(w1);
         compute_item(w0);
@@ -201,8 +203,10 @@ void launch_ng(const LinearArgs& a, cudaStream_t s) {
     }
     const int n_rb = (a.N + 15) / 16;
     const int grid = n_rb < resident ? n_rb : resident;
-    if (a.w_up) w4a4_mma_kernel<NG, true><<<grid, MMA_WARPS * 32, 0, s>>>(a);
-    else w4a4_mma_kernel<NG, false><<<grid, MMA_WARPS * 32, 0, s>>>(a);
+    cudaError_t e;
+    if (a.w_up) e = launch_dependent(w4a4_mma_kernel<NG, true>, dim3(grid), dim3(MMA_WARPS * 32), 0, s, a);
+    else e = launch_dependent(w4a4_mma_kernel<NG, false>, dim3(grid), dim3(MMA_WARPS * 32), 0, s, a);
+    if (e != cudaSuccess) note_cuda_error(e);
 }
 
 }  // namespace mmas
