@@ -245,8 +245,26 @@ __global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
     const int lane = threadIdx.x & 31;
     const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), W = gridDim.x * (blockDim.x >> 5);
     const int chunks = a.K / 32;
+    constexpr bool TWO = !SWIGLU;   // rows in flight per warp (the gated pair already streams two weight rows)
+    auto load_row = [&](const uint8_t* wbase, int n, uint4* wv) {
+        const uint4* row = reinterpret_cast<const uint4*>(wbase + static_cast<int64_t>(n) * (a.K / 2));
+#pragma unroll
+        for (int i = 0; i < CPL; ++i) {
+            const int c = lane + 32 * i;
+            wv[i] = c < chunks ? __ldg(row + c) : make_uint4(0, 0, 0, 0);   // zero weights meet zero activations
+        }
+    };
+    auto load_rows = [&](int n, uint4* g0, uint4* g1, uint4* u0) {
+        load_row(a.w, n, g0);
+        if (SWIGLU) load_row(a.w_up, n, u0);
+        if (TWO && n + W < a.N) load_row(a.w, n + W, g1);
+    };
+    // The first rows' weights do not depend on the kernel before this one (the quantizer): fetch them, then wait.
+    // (Not for the gated pair: holding three rows across the wait costs the registers of the third resident CTA.)
+    uint4 g0[CPL], g1[TWO ? CPL : 1], u0[SWIGLU ? CPL : 1];
+    if (!SWIGLU && gw < a.N) load_rows(gw, g0, g1, u0);
     pdl_launch_dependents();
-    pdl_wait();   // the activation row comes from the kernel before this one
+    pdl_wait();
     uint4 xl[CPL], xh[CPL];
 #pragma unroll
     for (int i = 0; i < CPL; ++i) {
@@ -278,14 +296,6 @@ __global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
         for (int off = 16; off > 0; off >>= 1) acc += __shfl_xor_sync(0xffffffffu, acc, off);
         return acc;
     };
-    auto load_row = [&](const uint8_t* wbase, int n, uint4* wv) {
-        const uint4* row = reinterpret_cast<const uint4*>(wbase + static_cast<int64_t>(n) * (a.K / 2));
-#pragma unroll
-        for (int i = 0; i < CPL; ++i) {
-            const int c = lane + 32 * i;
-            wv[i] = c < chunks ? __ldg(row + c) : make_uint4(0, 0, 0, 0);   // zero weights meet zero activations
-        }
-    };
     auto finish = [&](int n, int raw_g, int raw_u) {
         if (lane != 0) return;
         const int t = finish_acc(raw_g, bs);
@@ -293,14 +303,10 @@ __global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
         if (SWIGLU) y = swiglu(y, dequant(finish_acc(raw_u, bs), sx, __half2float(a.w_up_scales[n])));
         store_out(a.out, n, a.out_dtype, y, t);
     };
-    constexpr bool TWO = !SWIGLU;   // rows in flight per warp (the gated pair already streams two weight rows)
     for (int n = gw; n < a.N; n += (TWO ? 2 : 1) * W) {
         const int n2 = n + W;
         const bool two = TWO && n2 < a.N;
-        uint4 g0[CPL], g1[TWO ? CPL : 1], u0[SWIGLU ? CPL : 1];
-        load_row(a.w, n, g0);
-        if (SWIGLU) load_row(a.w_up, n, u0);
-        if (TWO && two) load_row(a.w, n2, g1);
+        if (SWIGLU || n != gw) load_rows(n, g0, g1, u0);
         finish(n, dot(g0), SWIGLU ? dot(u0) : 0);
         if (TWO && two) finish(n2, dot(g1), 0);
     }
