@@ -212,44 +212,74 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
         // 128-byte rows under the 128B TMA swizzle: 16-byte chunk c of row r sits at chunk c ^ (r & 7).
         // Consecutive rows then hit different banks for the same c, so the register a chunk lands in is fixed.
         const int sw = src_row & 7;
-        uint32_t it = 0;
-        int s = 0, j = 0, sd = 0;      // sd: slot of stage it - U
-        uint32_t ph = 0, phd = 0;
-        for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x) {
-            for (int ks = 0; ks < k_steps; ++ks, ++it) {
-                // weight tile j was last read by the MMAs of stage it - U, whose completion is that stage's done barrier
-                bool ok = mbar_wait(full(s), ph, abort_flag);
-                if (ok && it >= static_cast<uint32_t>(U)) {
-                    ok = mbar_wait(done(sd), phd, abort_flag);
-                    if (++sd == S) { sd = 0; phd ^= 1u; }
-                }
-                if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-                tc_fence_after();
+        const int my_tiles = static_cast<int>(blockIdx.x) < total_tiles
+                                 ? (total_tiles - 1 - static_cast<int>(blockIdx.x)) / static_cast<int>(gridDim.x) + 1 : 0;
+        const uint32_t total_its = static_cast<uint32_t>(my_tiles) * static_cast<uint32_t>(k_steps);
+        // One stage: packed row (shared memory) -> two ANDs per word -> tensor-memory weight tile j_.
+        auto unpack_stage = [&](int s_, int j_) {
 #pragma unroll
-                for (int h = 0; h < 2; ++h) {
-                    const uint8_t* src = sm + s * stage_bytes + src_row * 128;
-                    uint32_t r[32];   // column q holds codes k = 4q .. 4q+3 of this half of the row
+            for (int h = 0; h < 2; ++h) {
+                const uint8_t* src = sm + s_ * stage_bytes + src_row * 128;
+                uint32_t r[32];   // column q holds codes k = 4q .. 4q+3 of this half of the row
 #pragma unroll
-                    for (int c = 0; c < 4; ++c) {
-                        const uint4 v = *reinterpret_cast<const uint4*>(src + (((4 * h + c) ^ sw) << 4));
-                        r[4 * c + 0] = v.x & 0x0F0F0F0Fu; r[4 * c + 1] = v.y & 0x0F0F0F0Fu;      // codes 16c .. 16c+15 (+8)
-                        r[4 * c + 2] = v.z & 0x0F0F0F0Fu; r[4 * c + 3] = v.w & 0x0F0F0F0Fu;
-                        r[16 + 4 * c + 0] = v.x & 0xF0F0F0F0u; r[16 + 4 * c + 1] = v.y & 0xF0F0F0F0u;  // codes 64+16c .. (x16)
-                        r[16 + 4 * c + 2] = v.z & 0xF0F0F0F0u; r[16 + 4 * c + 3] = v.w & 0xF0F0F0F0u;
-                    }
-                    tc_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
-                                static_cast<uint32_t>(tmem_a_col + j * A_COLS + 32 * h), r);
+                for (int c = 0; c < 4; ++c) {
+                    const uint4 v = *reinterpret_cast<const uint4*>(src + (((4 * h + c) ^ sw) << 4));
+                    r[4 * c + 0] = v.x & 0x0F0F0F0Fu; r[4 * c + 1] = v.y & 0x0F0F0F0Fu;      // codes 16c .. 16c+15 (+8)
+                    r[4 * c + 2] = v.z & 0x0F0F0F0Fu; r[4 * c + 3] = v.w & 0x0F0F0F0Fu;
+                    r[16 + 4 * c + 0] = v.x & 0xF0F0F0F0u; r[16 + 4 * c + 1] = v.y & 0xF0F0F0F0u;  // codes 64+16c .. (x16)
+                    r[16 + 4 * c + 2] = v.z & 0xF0F0F0F0u; r[16 + 4 * c + 3] = v.w & 0xF0F0F0F0u;
                 }
-                tc_wait_st();
-                tc_fence_before();
-                __syncwarp();
-                if (lane == 0) {
-                    mbar_arrive(wp_empty(s));
-                    mbar_arrive(a_full(j));
-                }
-                if (++s == S) { s = 0; ph ^= 1u; }
-                if (++j == U) j = 0;
+                tc_st32(tmem_base + (static_cast<uint32_t>(quad * 32) << 16) +
+                            static_cast<uint32_t>(tmem_a_col + j_ * A_COLS + 32 * h), r);
             }
+        };
+        // With deep rings (narrow token tiles) two stages per round: every barrier operation costs this warp its
+        // latency (100-200 cycles even on a completed phase), so the four probes of a round are issued together and
+        // the two stages share one wait::st and one round of arrivals; with shallow rings that would hold two of three
+        // slots at once, so there a round is one stage. Stage it lives in slot it % S and weight tile it % U; weight
+        // tile j was last read by the MMAs of stage it - U, whose completion is that stage's done barrier (slot sd).
+        const bool pairwise = S >= 6 && U == U_MAX;
+        int s = 0, j = 0, sd = 0;
+        uint32_t ph = 0, phd = 0;
+        for (uint32_t it = 0; it < total_its && !failed; it += pairwise ? 2u : 1u) {
+            const bool two = pairwise && it + 1 < total_its;
+            const int s1 = s + 1 == S ? 0 : s + 1, j1 = j + 1;          // pairwise: U is even and j stays even
+            const uint32_t ph1 = s + 1 == S ? ph ^ 1u : ph;
+            const bool need_done = it >= static_cast<uint32_t>(U);      // then also for stage it + 1
+            const int sd1 = sd + 1 == S ? 0 : sd + 1;
+            const uint32_t phd1 = sd + 1 == S ? phd ^ 1u : phd;
+            const bool f0 = mbar_test_wait(full(s), ph);
+            const bool f1 = !two || mbar_test_wait(full(s1), ph1);
+            const bool d0 = !need_done || mbar_test_wait(done(sd), phd);
+            const bool d1 = !need_done || !two || mbar_test_wait(done(sd1), phd1);
+            bool ok = f0 || mbar_wait(full(s), ph, abort_flag);
+            ok = ok && (f1 || mbar_wait(full(s1), ph1, abort_flag));
+            ok = ok && (d0 || mbar_wait(done(sd), phd, abort_flag));
+            ok = ok && (d1 || mbar_wait(done(sd1), phd1, abort_flag));
+            if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+            tc_fence_after();
+            unpack_stage(s, j);
+            if (two) unpack_stage(s1, j1);
+            tc_wait_st();
+            tc_fence_before();
+            __syncwarp();
+            if (lane == 0) {
+                mbar_arrive(wp_empty(s));
+                mbar_arrive(a_full(j));
+                if (two) {
+                    mbar_arrive(wp_empty(s1));
+                    mbar_arrive(a_full(j1));
+                }
+            }
+            const int adv = pairwise ? 2 : 1;
+            if (need_done) {
+                sd += adv;
+                if (sd >= S) { sd -= S; phd ^= 1u; }
+            }
+            s += adv;
+            if (s >= S) { s -= S; ph ^= 1u; }
+            j += adv;
+            if (j >= U) j = 0;
         }
     } else {
         // ---------------- epilogue warps: warp % 4 selects the 32-lane quadrant of tensor memory
