@@ -715,12 +715,13 @@ def run_single_kernel(args):
     if args.kernel == "quantize":
         for i in range(args.steps):
             B.sqap_quantize_act(x, M, H, H, None, B.SQAP_Q_ROTATE if i % 2 == 0 else 0, q, sx)
-    elif args.kernel in ("gemm", "gemv", "stream", "swiglu"):
-        names = {"gemm": ("qkv",), "gemv": ("qkv",), "stream": ("qkv",), "swiglu": ("gate", "up")}[args.kernel]
+    elif args.kernel in ("gemm", "gemv", "stream", "midm", "swiglu"):
+        names = {"gemm": ("qkv",), "gemv": ("qkv",), "stream": ("qkv",), "midm": ("o",), "swiglu": ("gate", "up")}[args.kernel]
         wts = wl.config4_weights(seed=4)
         ws = [B.sqap_pack_weights(np.ascontiguousarray(wts[n + "_codes"]), np.ascontiguousarray(wts[n + "_scales"]),
                                   wts[n + "_codes"].shape[0], H) for n in names]
-        Mk = {"gemv": 1, "stream": N_OBS}.get(args.kernel, M)   # stream: one decode token per observation
+        # stream: one decode token per observation; midm: one observation pruned to 160 rows (O projection)
+        Mk = {"gemv": 1, "stream": N_OBS, "midm": 160}.get(args.kernel, M)
         N = ws[0].N
         out = torch.empty(Mk, N, dtype=torch.float16, device=dev)
         nb = B.sqap_workspace_bytes(Mk, N, H)
@@ -756,7 +757,7 @@ def main():
                     help="time every kernel of the path alone at the workload's shapes (one JSON table, no bench line)")
     ap.add_argument("--stack", action="store_true",
                     help="time configs[3] (32-layer stack: prefill + 7 decode tokens for one observation); own JSON line")
-    ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "stream", "quantize", "prune"],
+    ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "stream", "midm", "quantize", "prune"],
                     help="profiling aid: launch only this kernel --steps times (no bench line)")
     args = ap.parse_args()
     if args.stack:
