@@ -240,8 +240,15 @@ __global__ void __launch_bounds__(256) w4a4_gemv_kernel(LinearArgs a) {
 // 16-byte weight chunks (lane, lane + 32, ...) of whatever row its warp streams, so it loads the 2 x 16
 // activation bytes that go with each of them once and then only streams weights: two rows at a time (all their
 // loads issued before the first dp4a), persistent warps striding over the output channels.
-template <bool SWIGLU, int CPL>
+// FUSEQ: the kernel also quantizes the row (plain per-token quantizer, no rotation): every CTA repeats the small
+// job (one 16-byte chunk or two per thread, two block-wide reductions) into shared memory while its first weight
+// rows are in flight, which takes a whole kernel out of a decode step's chain; CTA 0 also leaves the expanded codes,
+// their sum and the scale in the workspace, as the separate quantizer would have.
+template <bool SWIGLU, int CPL, bool FUSEQ>
 __global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
+    __shared__ __align__(16) int8_t xs[FUSEQ ? 32 * 32 * CPL : 16];
+    __shared__ float red_f[8];
+    __shared__ int red_i[8];
     const int lane = threadIdx.x & 31;
     const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), W = gridDim.x * (blockDim.x >> 5);
     const int chunks = a.K / 32;
@@ -265,6 +272,71 @@ __global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
     if (!SWIGLU && gw < a.N) load_rows(gw, g0, g1, u0);
     pdl_launch_dependents();
     pdl_wait();
+    int bs;
+    float sx;
+    if (FUSEQ) {
+        // the quantizer of quantize.cu for one row: max-abs, scale = amax / 7, inv = 7 / amax, codes by the magic add
+        const int tid = threadIdx.x, wid = tid >> 5, n8 = a.K / 8;   // n8 <= 2 * 256 chunks of eight values
+        const int64_t src = a.fuse_row_index ? static_cast<int64_t>(a.fuse_row_index[0]) : 0;
+        const uint4* xr = reinterpret_cast<const uint4*>(a.fuse_x + src * a.fuse_ldx);
+        uint4 c8[2];
+        float amax = 0.0f;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int c = tid + 256 * i;
+            c8[i] = make_uint4(0, 0, 0, 0);
+            if (c < n8) {
+                c8[i] = __ldg(xr + c);
+                const __half2* h = reinterpret_cast<const __half2*>(&c8[i]);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    const float2 f = __half22float2(__habs2(h[q]));
+                    amax = fmaxf(amax, fmaxf(f.x, f.y));
+                }
+            }
+        }
+        amax = warp_max(amax);
+        if (lane == 0) red_f[wid] = amax;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < 8; ++w) amax = fmaxf(amax, red_f[w]);
+        float inv;
+        scale_of(amax, sx, inv);
+        int bias = 0;
+#pragma unroll
+        for (int i = 0; i < 2; ++i) {
+            const int c = tid + 256 * i;
+            if (c < n8) {
+                uint64_t p[4];
+                uint32_t t[8];
+                half8_to_pairs(c8[i], p);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) round_pair(p[q], inv, MAGIC, t[2 * q], t[2 * q + 1]);
+                uint32_t w0 = low_bytes(t[0], t[1], t[2], t[3]), w1 = low_bytes(t[4], t[5], t[6], t[7]);
+                if (((8 * c) % (2 * a.half)) < a.half) {   // these codes meet low weight nibbles
+                    bias = __dp4a(static_cast<int>(w0), 0x01010101, bias);
+                    bias = __dp4a(static_cast<int>(w1), 0x01010101, bias);
+                    w0 = times16(w0);
+                    w1 = times16(w1);
+                }
+                reinterpret_cast<uint2*>(xs)[c] = make_uint2(w0, w1);
+                if (blockIdx.x == 0) reinterpret_cast<uint2*>(const_cast<int8_t*>(a.x8))[c] = make_uint2(w0, w1);
+            }
+        }
+        bias = warp_sum(bias);
+        if (lane == 0) red_i[wid] = bias;
+        __syncthreads();   // also: xs is complete
+        bs = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) bs += red_i[w];
+        if (blockIdx.x == 0 && tid == 0) {
+            const_cast<int32_t*>(a.bias_sum)[0] = bs;
+            const_cast<float*>(a.act_scales)[0] = sx;
+        }
+    } else {
+        bs = a.bias_sum[0];
+        sx = a.act_scales[0];
+    }
     uint4 xl[CPL], xh[CPL];
 #pragma unroll
     for (int i = 0; i < CPL; ++i) {
@@ -273,12 +345,15 @@ __global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
         if (c < chunks) {
             int lo_k, hi_k;
             chunk_k(c, a.half, lo_k, hi_k);
-            xl[i] = __ldg(reinterpret_cast<const uint4*>(a.x8 + lo_k));
-            xh[i] = __ldg(reinterpret_cast<const uint4*>(a.x8 + hi_k));
+            if (FUSEQ) {
+                xl[i] = *reinterpret_cast<const uint4*>(xs + lo_k);
+                xh[i] = *reinterpret_cast<const uint4*>(xs + hi_k);
+            } else {
+                xl[i] = __ldg(reinterpret_cast<const uint4*>(a.x8 + lo_k));
+                xh[i] = __ldg(reinterpret_cast<const uint4*>(a.x8 + hi_k));
+            }
         }
     }
-    const int bs = a.bias_sum[0];
-    const float sx = a.act_scales[0];
     auto dot = [&](const uint4* wv) {
         int acc = 0;
 #pragma unroll
@@ -324,8 +399,13 @@ static void launch_gemv1(const LinearArgs& a, cudaStream_t s) {
     const int need = (a.N + 7) / 8;
     const int grid = need < blocks ? need : blocks;
     cudaError_t e;
-    if (a.w_up) e = launch_dependent(w4a4_gemv1_kernel<true, CPL>, dim3(grid), dim3(256), 0, s, a);
-    else e = launch_dependent(w4a4_gemv1_kernel<false, CPL>, dim3(grid), dim3(256), 0, s, a);
+    if (a.fuse_x) {
+        if (a.w_up) e = launch_dependent(w4a4_gemv1_kernel<true, CPL, true>, dim3(grid), dim3(256), 0, s, a);
+        else e = launch_dependent(w4a4_gemv1_kernel<false, CPL, true>, dim3(grid), dim3(256), 0, s, a);
+    } else {
+        if (a.w_up) e = launch_dependent(w4a4_gemv1_kernel<true, CPL, false>, dim3(grid), dim3(256), 0, s, a);
+        else e = launch_dependent(w4a4_gemv1_kernel<false, CPL, false>, dim3(grid), dim3(256), 0, s, a);
+    }
     if (e != cudaSuccess) note_cuda_error(e);
 }
 
@@ -380,6 +460,9 @@ static LinearArgs make_args(void* workspace, const float* act_scales, int M, con
     a.out = out;
     a.ldo = ldo;
     a.out_dtype = out_dtype;
+    a.fuse_x = nullptr;
+    a.fuse_ldx = 0;
+    a.fuse_row_index = nullptr;
     return a;
 }
 
@@ -500,10 +583,17 @@ sqap_status sqap_quantize_linear(const void* x, int M, int64_t ldx, const int32_
     cudaStream_t s = static_cast<cudaStream_t>(stream);
 
     float* scales = reinterpret_cast<float*>(static_cast<uint8_t*>(workspace) + sqap_workspace_bytes(M, w->N, w->K, 0));
-    const LinearArgs a = make_args(workspace, scales, M, w, w_up, out, ldo, out_dtype);
+    LinearArgs a = make_args(workspace, scales, M, w, w_up, out, ldo, out_dtype);
     LinearPath path;
     st = pick_path(a, lflags, &path);
     if (st != SQAP_OK) return st;
+    if (path == PATH_GEMV && M == 1 && a.K / 32 <= 32 * 4 && !(qflags & SQAP_Q_ROTATE)) {
+        // one row, no rotation: the streamer quantizes the row itself (one kernel instead of two)
+        a.fuse_x = static_cast<const __half*>(x);
+        a.fuse_ldx = ldx;
+        a.fuse_row_index = row_index;
+        return run_gemm(a, path, s);
+    }
     st = quantize_expanded(static_cast<const __half*>(x), M, a.K, ldx, row_index, qflags, a.half,
                            const_cast<int8_t*>(a.x8), const_cast<int32_t*>(a.bias_sum), scales, s);
     if (st != SQAP_OK) return st;

@@ -21,6 +21,12 @@ struct LinearArgs {
     void* out;
     int64_t ldo;
     int out_dtype;
+    // Set only when the kernel itself is to quantize the (single) activation row: the fp16 source, as in
+    // sqap_quantize_act; x8 / bias_sum / act_scales above are then OUTPUTS (written once, for later calls that
+    // reuse the expanded form), not inputs.
+    const __half* fuse_x;
+    int64_t fuse_ldx;
+    const int32_t* fuse_row_index;
 };
 
 __device__ __forceinline__ int finish_acc(int raw, int bias_sum) { return (raw - 128 * bias_sum) >> 4; }

@@ -21,9 +21,6 @@
 namespace sqap {
 
 constexpr int SINK_NIBBLES = 0, SINK_EXPANDED = 1;
-constexpr float MAGIC = 12582912.0f;   // 1.5 * 2^23: low byte of fl(y + MAGIC) = code as int8
-constexpr float MAGIC8 = 12582920.0f;  // MAGIC + 8:  low nibble of fl(y + MAGIC8) = code + 8 (0..15)
-
 struct QuantOut {
     uint8_t* q;         // SINK_NIBBLES: [M][K/2]
     int8_t* x8;         // SINK_EXPANDED: [M][K]
@@ -33,12 +30,6 @@ struct QuantOut {
 };
 
 // ------------------------------------------------------------------------------- packed fp32 helpers
-__device__ __forceinline__ uint64_t pk(float lo, float hi) {
-    uint64_t r;
-    asm("mov.b64 %0, {%1, %2};" : "=l"(r) : "f"(lo), "f"(hi));
-    return r;
-}
-__device__ __forceinline__ void upk(uint64_t p, float& lo, float& hi) { asm("mov.b64 {%0, %1}, %2;" : "=f"(lo), "=f"(hi) : "l"(p)); }
 __device__ __forceinline__ void upk_bits(uint64_t p, uint32_t& lo, uint32_t& hi) { asm("mov.b64 {%0, %1}, %2;" : "=r"(lo), "=r"(hi) : "l"(p)); }
 __device__ __forceinline__ uint64_t add2(uint64_t a, uint64_t b) {
     uint64_t d;
@@ -49,17 +40,6 @@ __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
     uint64_t d;
     asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
-}
-
-__device__ __forceinline__ float warp_max(float v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v = fmaxf(v, __shfl_xor_sync(0xffffffffu, v, o));
-    return v;
-}
-__device__ __forceinline__ int warp_sum(int v) {
-#pragma unroll
-    for (int o = 16; o > 0; o >>= 1) v += __shfl_xor_sync(0xffffffffu, v, o);
-    return v;
 }
 
 // Block-wide max of non-negative values; every thread gets the result. red: >= 32 floats of smem.
@@ -86,37 +66,11 @@ __device__ __forceinline__ int block_sum(int v, int* red) {
     return r;
 }
 
-__device__ __forceinline__ void scale_of(float amax, float& scale, float& inv) {
-    scale = 1.0f;
-    inv = 0.0f;
-    if (amax != 0.0f) {
-        scale = __fdiv_rn(amax, 7.0f);
-        inv = __fdiv_rn(7.0f, amax);
-    }
-}
-
-// Bits of fl(fl(v * inv) + magic) for a pair of values. The product must be rounded to fp32 before the sum
-// (a fused multiply-add rounds once and lands on the other side of a tie): scalar __fmul_rn / __fadd_rn are
-// never contracted, whereas a packed multiply followed by a packed add was seen to be.
-__device__ __forceinline__ void round_pair(uint64_t v, float inv, float magic, uint32_t& lo, uint32_t& hi) {
-    float a, b;
-    upk(v, a, b);
-    lo = __float_as_uint(__fadd_rn(__fmul_rn(a, inv), magic));
-    hi = __float_as_uint(__fadd_rn(__fmul_rn(b, inv), magic));
-}
-
-// Low bytes of four words -> one word.
-__device__ __forceinline__ uint32_t low_bytes(uint32_t t0, uint32_t t1, uint32_t t2, uint32_t t3) {
-    return __byte_perm(__byte_perm(t0, t1, 0x0040), __byte_perm(t2, t3, 0x0040), 0x5410);
-}
 // Two words of four bytes each holding code + 8 (0..15) -> eight two's-complement nibbles, value i in nibble i.
 __device__ __forceinline__ uint32_t nibbles_of(uint32_t w0, uint32_t w1) {
     const uint32_t x0 = w0 | (w0 >> 4), x1 = w1 | (w1 >> 4);
     return __byte_perm(x0, x1, 0x6420) ^ 0x88888888u;
 }
-// A word of four int8 codes -> the same codes times 16 (each still fits a byte).
-__device__ __forceinline__ uint32_t times16(uint32_t w) { return (w << 4) & 0xF0F0F0F0u; }
-
 // Eight consecutive values (k = 8c .. 8c+7 of the row) -> output. v as four packed pairs.
 template <int SINK>
 __device__ __forceinline__ void emit_chunk(const uint64_t* v, float inv, int c, const QuantOut& o, int64_t row,
@@ -137,15 +91,6 @@ __device__ __forceinline__ void emit_chunk(const uint64_t* v, float inv, int c, 
             out = make_uint2(times16(w0), times16(w1));
         }
         reinterpret_cast<uint2*>(o.x8 + row * K)[c] = out;
-    }
-}
-
-__device__ __forceinline__ void half8_to_pairs(const uint4& u, uint64_t* p) {
-    const __half2* h = reinterpret_cast<const __half2*>(&u);
-#pragma unroll
-    for (int i = 0; i < 4; ++i) {
-        const float2 f = __half22float2(h[i]);
-        p[i] = pk(f.x, f.y);
     }
 }
 

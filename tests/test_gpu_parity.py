@@ -343,6 +343,32 @@ def test_linear_dispatch_boundaries(M, N, K, swiglu):
     check_linear(x, g[0], g[1], up=u, flags_list=[0, B.SQAP_L_FORCE_SIMT])
 
 
+@pytest.mark.parametrize("M,rotate", [(1, False), (1, True), (5, False), (40, False)])
+def test_fused_call_leaves_the_expanded_activations_for_reuse(M, rotate):
+    """After sqap_quantize_linear the workspace holds the expanded codes, the row sums and (behind them) the
+    scales of those activations: a second weight matrix applied with SQAP_L_REUSE_EXPANDED must give exactly what
+    the full call gives. M = 1 without rotation is the case where the streamer quantizes the row itself."""
+    K, N = 4096, 264
+    x = wl.activations(30, M + 7, M, K, 41, 30.0)
+    w1 = G.pack(wl.weight_codes(30, 1, N, K), wl.weight_scales(30, 1, N, mult=0.25))
+    w2 = G.pack(wl.weight_codes(30, 2, N, K), wl.weight_scales(30, 2, N, mult=0.25))
+    ref2 = G.quantize_linear(x, w2, rotate=rotate)
+    xd = torch.from_numpy(np.ascontiguousarray(x)).to("cuda")
+    nb = B.sqap_quantize_linear_workspace_bytes(M, N, K)
+    ws = torch.empty(nb, dtype=torch.uint8, device="cuda")
+    out1 = torch.empty(M, N, dtype=torch.float16, device="cuda")
+    out2 = torch.empty(M, N, dtype=torch.float16, device="cuda")
+    B.sqap_quantize_linear(xd, M, K, None, B.SQAP_Q_ROTATE if rotate else 0, w1, None, out1, N, B.SQAP_FP16, 0, ws, nb)
+    dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    scales_ptr = ws.data_ptr() + B.sqap_workspace_bytes(M, N, K)
+    B.sqap_w4a4_linear(dummy, scales_ptr, M, w2, None, out2, N, B.SQAP_FP16, B.SQAP_L_REUSE_EXPANDED, ws, nb)
+    torch.cuda.synchronize()
+    assert B.sqap_device_status() == B.SQAP_OK
+    assert np.array_equal(out2.cpu().numpy().view(np.uint16), ref2)
+    w1.close()
+    w2.close()
+
+
 def test_linear_special_operands():
     K = N = 256
     x = wl.activations(22, 1, 16, K, 3, 20.0)
