@@ -587,7 +587,8 @@ sqap_status sqap_quantize_linear(const void* x, int M, int64_t ldx, const int32_
     LinearPath path;
     st = pick_path(a, lflags, &path);
     if (st != SQAP_OK) return st;
-    if (path == PATH_GEMV && M == 1 && a.K / 32 <= 32 * 4 && !(qflags & SQAP_Q_ROTATE)) {
+    const bool one_plain_row = M == 1 && !(qflags & SQAP_Q_ROTATE);
+    if (one_plain_row && ((path == PATH_GEMV && a.K / 32 <= 32 * 4) || (path == PATH_MMA && a.K <= MMA_FUSE_MAX_K))) {
         // one row, no rotation: the streamer quantizes the row itself (one kernel instead of two)
         a.fuse_x = static_cast<const __half*>(x);
         a.fuse_ldx = ldx;

@@ -55,6 +55,7 @@ sqap_status launch_linear_tcgen05_pair(const LinearArgs& a, cudaStream_t s);
 
 // Register-MMA weight streamer for a handful of tokens (linear_mma.cu): K % 128 == 0 and M <= MMA_STREAM_MAX_M.
 constexpr int MMA_STREAM_MAX_M = 32;
+constexpr int MMA_FUSE_MAX_K = 16384;   // longest single row it will quantize itself (K bytes of shared memory)
 bool mma_stream_supports(const LinearArgs& a);
 sqap_status launch_linear_mma_stream(const LinearArgs& a, cudaStream_t s);
 

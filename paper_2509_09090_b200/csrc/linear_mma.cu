@@ -18,6 +18,7 @@
 // 16t and 64+16t of the block. Four MMAs per block and token group: (words 0,1 low), (2,3 low), (0,1 high),
 // (2,3 high).
 #include "linear.cuh"
+#include "quantize.cuh"
 
 namespace sqap {
 
@@ -63,8 +64,16 @@ struct ItemWeights {
 };
 
 // NG = token groups of 8 (M <= 8 * NG). Persistent: CTA c takes row blocks c, c + gridDim.x, ...
-template <int NG, bool SWIGLU>
+// FUSEQ (one row only): the kernel quantizes the activation row itself, as the single-row streamer of linear.cu
+// does: every CTA repeats the plain per-token quantizer into (dynamic) shared memory, K bytes, while its first
+// weights are in flight; CTA 0 also writes the expanded form to the workspace.
+template <int NG, bool SWIGLU, bool FUSEQ = false>
 __global__ void __launch_bounds__(MMA_WARPS * 32, 2) w4a4_mma_kernel(LinearArgs a) {
+    extern __shared__ __align__(16) int8_t xs[];   // FUSEQ: the expanded codes of the row
+    __shared__ float q_red_f[MMA_WARPS];
+    __shared__ int q_red_i[MMA_WARPS];
+    __shared__ int q_bias;
+    __shared__ float q_scale;
     constexpr int SETS = SWIGLU ? 2 : 1;
     constexpr int KU = SWIGLU ? (NG <= 2 ? 2 : 1) : (NG <= 2 ? 4 : 2);
     __shared__ int red[MMA_WARPS][SETS * NG * 4][32];
@@ -133,8 +142,13 @@ __global__ void __launch_bounds__(MMA_WARPS * 32, 2) w4a4_mma_kernel(LinearArgs 
                 for (int j = 0; j < NG; ++j) {
                     xl[j] = xh[j] = make_uint4(0, 0, 0, 0);   // tokens past M contribute zeros
                     if (xok[j]) {
-                        xl[j] = __ldg(xp[j] + 8 * b);
-                        xh[j] = __ldg(xp[j] + 8 * b + 4);
+                        if (FUSEQ) {   // one row: token 0 only
+                            xl[j] = *reinterpret_cast<const uint4*>(xs + 128 * b + 16 * t);
+                            xh[j] = *reinterpret_cast<const uint4*>(xs + 128 * b + 64 + 16 * t);
+                        } else {
+                            xl[j] = __ldg(xp[j] + 8 * b);
+                            xh[j] = __ldg(xp[j] + 8 * b + 4);
+                        }
                     }
                 }
                 block_mma<NG>(acc, w.a[u], w.b[u], xl, xh);
@@ -166,8 +180,8 @@ __global__ void __launch_bounds__(MMA_WARPS * 32, 2) w4a4_mma_kernel(LinearArgs 
                 if (SWIGLU) raw_u += red[w8][NG * 4 + idx][ln];
             }
             if (n < a.N && m < a.M) {
-                const int bs = a.bias_sum[m];
-                const float sx = a.act_scales[m];
+                const int bs = FUSEQ ? q_bias : a.bias_sum[m];
+                const float sx = FUSEQ ? q_scale : a.act_scales[m];
                 const int tq = finish_acc(raw, bs);
                 float y = dequant(tq, sx, __half2float(a.w_scales[n]));
                 if (SWIGLU) y = swiglu(y, dequant(finish_acc(raw_u, bs), sx, __half2float(a.w_up_scales[n])));
@@ -183,6 +197,63 @@ __global__ void __launch_bounds__(MMA_WARPS * 32, 2) w4a4_mma_kernel(LinearArgs 
     if (total_items > 0) load_item(w0);
     pdl_launch_dependents();
     pdl_wait();   // the activations come from the kernel before this one; the weights above do not
+    if (FUSEQ) {
+        // the quantizer of quantize.cu for one row (two passes over it, the second from cache): max-abs,
+        // scale = amax / 7, inv = 7 / amax, codes by the magic add; half = 64 here (K % 128 == 0)
+        const int tid = threadIdx.x, n8 = a.K / 8;
+        const int64_t src = a.fuse_row_index ? static_cast<int64_t>(a.fuse_row_index[0]) : 0;
+        const uint4* xr = reinterpret_cast<const uint4*>(a.fuse_x + src * a.fuse_ldx);
+        float amax = 0.0f;
+        for (int c = tid; c < n8; c += MMA_WARPS * 32) {
+            const uint4 v = __ldg(xr + c);
+            const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float2 f = __half22float2(__habs2(h[q]));
+                amax = fmaxf(amax, fmaxf(f.x, f.y));
+            }
+        }
+        amax = warp_max(amax);
+        if (lane == 0) q_red_f[warp] = amax;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < MMA_WARPS; ++w) amax = fmaxf(amax, q_red_f[w]);
+        float scale, inv;
+        scale_of(amax, scale, inv);
+        int bias = 0;
+        for (int c = tid; c < n8; c += MMA_WARPS * 32) {
+            const uint4 v = __ldg(xr + c);
+            uint64_t p[4];
+            uint32_t tt[8];
+            half8_to_pairs(v, p);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) round_pair(p[q], inv, MAGIC, tt[2 * q], tt[2 * q + 1]);
+            uint32_t w0 = low_bytes(tt[0], tt[1], tt[2], tt[3]), w1 = low_bytes(tt[4], tt[5], tt[6], tt[7]);
+            if (((8 * c) & 127) < 64) {   // these codes meet low weight nibbles
+                bias = __dp4a(static_cast<int>(w0), 0x01010101, bias);
+                bias = __dp4a(static_cast<int>(w1), 0x01010101, bias);
+                w0 = times16(w0);
+                w1 = times16(w1);
+            }
+            reinterpret_cast<uint2*>(xs)[c] = make_uint2(w0, w1);
+            if (blockIdx.x == 0) reinterpret_cast<uint2*>(const_cast<int8_t*>(a.x8))[c] = make_uint2(w0, w1);
+        }
+        bias = warp_sum(bias);
+        if (lane == 0) q_red_i[warp] = bias;
+        __syncthreads();   // also: xs is complete
+        if (tid == 0) {
+            int total = 0;
+#pragma unroll
+            for (int w = 0; w < MMA_WARPS; ++w) total += q_red_i[w];
+            q_bias = total;
+            q_scale = scale;
+            if (blockIdx.x == 0) {
+                const_cast<int32_t*>(a.bias_sum)[0] = total;
+                const_cast<float*>(a.act_scales)[0] = scale;
+            }
+        }
+        // q_bias / q_scale are read only after the __syncthreads of a row block's reduction
+    }
     for (int i = 0; i < total_items; i += 2) {
         if (i + 1 < total_items) load_item(w1);
         compute_item(w0);
@@ -204,7 +275,11 @@ void launch_ng(const LinearArgs& a, cudaStream_t s) {
     const int n_rb = (a.N + 15) / 16;
     const int grid = n_rb < resident ? n_rb : resident;
     cudaError_t e;
-    if (a.w_up) e = launch_dependent(w4a4_mma_kernel<NG, true>, dim3(grid), dim3(MMA_WARPS * 32), 0, s, a);
+    if (NG == 1 && a.fuse_x) {
+        const size_t smem = static_cast<size_t>(a.K);   // <= MMA_FUSE_MAX_K: within the default dynamic limit
+        if (a.w_up) e = launch_dependent(w4a4_mma_kernel<1, true, true>, dim3(grid), dim3(MMA_WARPS * 32), smem, s, a);
+        else e = launch_dependent(w4a4_mma_kernel<1, false, true>, dim3(grid), dim3(MMA_WARPS * 32), smem, s, a);
+    } else if (a.w_up) e = launch_dependent(w4a4_mma_kernel<NG, true>, dim3(grid), dim3(MMA_WARPS * 32), 0, s, a);
     else e = launch_dependent(w4a4_mma_kernel<NG, false>, dim3(grid), dim3(MMA_WARPS * 32), 0, s, a);
     if (e != cudaSuccess) note_cuda_error(e);
 }

@@ -343,13 +343,15 @@ def test_linear_dispatch_boundaries(M, N, K, swiglu):
     check_linear(x, g[0], g[1], up=u, flags_list=[0, B.SQAP_L_FORCE_SIMT])
 
 
-@pytest.mark.parametrize("M,rotate", [(1, False), (1, True), (5, False), (40, False)])
-def test_fused_call_leaves_the_expanded_activations_for_reuse(M, rotate):
+@pytest.mark.parametrize("M,K,rotate", [(1, 4096, False), (1, 4096, True), (1, 11008, False), (1, 384, False),
+                                        (5, 4096, False), (40, 4096, False)])
+def test_fused_call_leaves_the_expanded_activations_for_reuse(M, K, rotate):
     """After sqap_quantize_linear the workspace holds the expanded codes, the row sums and (behind them) the
     scales of those activations: a second weight matrix applied with SQAP_L_REUSE_EXPANDED must give exactly what
-    the full call gives. M = 1 without rotation is the case where the streamer quantizes the row itself."""
-    K, N = 4096, 264
-    x = wl.activations(30, M + 7, M, K, 41, 30.0)
+    the full call gives. M = 1 without rotation is the case where the streamers quantize the row themselves (the
+    dp4a one up to 4096 codes, the register-MMA one beyond)."""
+    N = 264
+    x = wl.activations(30, M + 7, M, K, max(1, K // 100), 30.0)
     w1 = G.pack(wl.weight_codes(30, 1, N, K), wl.weight_scales(30, 1, N, mult=0.25))
     w2 = G.pack(wl.weight_codes(30, 2, N, K), wl.weight_scales(30, 2, N, mult=0.25))
     ref2 = G.quantize_linear(x, w2, rotate=rotate)
