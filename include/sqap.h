@@ -279,6 +279,17 @@ sqap_status sqap_project_center(const double Kmat[9], const double Rt[12], const
  * device set when one of their bounded waits runs out (SQAP_ERR_TIMEOUT) — SQAP_OK otherwise. */
 sqap_status sqap_device_status(void* stream);
 
+/*
+ * Self-test of the bounded waits (the paper has no counterpart; this is the library's own failure-detection
+ * mechanism). Every wait on a barrier inside the tensor-core kernels gives up after a fixed number of clocks,
+ * records SQAP_ERR_TIMEOUT in the device status word, drains and returns. This call launches one warp that runs that
+ * same wait, with the limit `limit_clocks` (1e3 .. 2e8 SM clocks, i.e. at most about 0.1 s), on a barrier nothing
+ * will ever arrive on. Afterwards sqap_device_status(stream) must return SQAP_ERR_TIMEOUT once and SQAP_OK on the next
+ * call, and the device stays fully usable. Touches no caller memory. Errors: INVALID (limit out of range),
+ * UNSUPPORTED (not an sm_100 device), CUDA.
+ */
+sqap_status sqap_selftest_bounded_wait(int64_t limit_clocks, void* stream);
+
 /* cudaError_t of the most recent failing CUDA call on this thread (0 if none). */
 int sqap_last_cuda_error(void);
 

@@ -26,7 +26,7 @@ EXPORTS = ("sqap_pack_weights", "sqap_quantize_weights", "sqap_free_weights", "s
            "sqap_quantize_linear", "sqap_quantize_linear_workspace_bytes",
            "sqap_prune_tokens", "sqap_attention_scores",
            "sqap_project_center", "sqap_device_status", "sqap_last_cuda_error", "sqap_status_string",
-           "sqap_kernel_launch_count")
+           "sqap_kernel_launch_count", "sqap_selftest_bounded_wait")
 
 
 class SqapError(RuntimeError):
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
                                                                               ctypes.POINTER(ctypes.c_int32),
                                                                               ctypes.POINTER(i32)]
     L.sqap_device_status.argtypes = [vp]
+    L.sqap_selftest_bounded_wait.argtypes = [i64, vp]
     L.sqap_last_cuda_error.restype = i32
     L.sqap_status_string.argtypes = [i32]
     L.sqap_status_string.restype = ctypes.c_char_p
@@ -232,6 +233,10 @@ def sqap_project_center(Kmat, Rt, xyz, patch_w: float, patch_h: float):
 
 def sqap_device_status(stream=None) -> int:
     return int(lib().sqap_device_status(_stream(stream)))
+
+
+def sqap_selftest_bounded_wait(limit_clocks: int, stream=None):
+    _check(lib().sqap_selftest_bounded_wait(limit_clocks, _stream(stream)), "sqap_selftest_bounded_wait")
 
 
 def sqap_kernel_launch_count() -> int:

@@ -24,14 +24,40 @@ sqap_status check_launch() {
     return SQAP_OK;
 }
 
-int* device_status_word() {
-    int* p = nullptr;
-    cudaError_t e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p), g_device_status);
-    if (e != cudaSuccess) {
-        note_cuda_error(e);
+static PerDevice<DeviceProps> g_props;
+
+const DeviceProps* device_props() {
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) {
+        cudaGetLastError();
         return nullptr;
     }
-    return p;
+    const DeviceProps* props = nullptr;
+    const sqap_status st = g_props.run(
+        [dev](DeviceProps* p) {
+            cudaError_t e = cudaDeviceGetAttribute(&p->sms, cudaDevAttrMultiProcessorCount, dev);
+            if (e == cudaSuccess) e = cudaDeviceGetAttribute(&p->cc_major, cudaDevAttrComputeCapabilityMajor, dev);
+            // in host code the symbol's name is not a device address: ask for it, with this device current
+            if (e == cudaSuccess) e = cudaGetSymbolAddress(reinterpret_cast<void**>(&p->status_word), g_device_status);
+            if (e != cudaSuccess) {
+                note_cuda_error(e);
+                cudaGetLastError();
+                return SQAP_ERR_CUDA;
+            }
+            return SQAP_OK;
+        },
+        &props);
+    return st == SQAP_OK ? props : nullptr;
+}
+
+int sm_count() {
+    const DeviceProps* p = device_props();
+    return (p && p->sms > 0) ? p->sms : 148;
+}
+
+int* device_status_word() {
+    const DeviceProps* p = device_props();
+    return p ? p->status_word : nullptr;
 }
 
 }  // namespace sqap

@@ -6,6 +6,8 @@
 #include <cuda_bf16.h>
 #include <stdint.h>
 
+#include <mutex>
+
 #include "../../include/sqap.h"
 
 namespace sqap {
@@ -18,6 +20,59 @@ sqap_status check_launch();  // cudaGetLastError -> status
 // Pointer to the device status word of the current device (set by kernels whose bounded waits expire).
 int* device_status_word();
 
+// What the launch code needs to know about a device, looked up once per device (api.cu; thread-safe).
+constexpr int MAX_DEVICES = 64;
+struct DeviceProps {
+    int sms;           // multiprocessors
+    int cc_major;      // compute capability, major
+    int* status_word;  // device address of the status word
+};
+// Properties of the CURRENT device; nullptr if it cannot be queried (or its ordinal is >= MAX_DEVICES).
+const DeviceProps* device_props();
+// Multiprocessor count of the current device (148 if it cannot be queried).
+int sm_count();
+
+// Set-up that has to happen once per DEVICE rather than once per process (function attributes such as the
+// dynamic shared-memory limit apply to the device that is current when they are set; occupancy figures differ
+// between devices). run() calls fn(&value) the first time it is used with a given device current, under a lock,
+// keeps the value it produced and from then on hands out a pointer to it (the value never changes again).
+template <typename T>
+class PerDevice {
+public:
+    template <typename F>
+    sqap_status run(F fn, const T** out = nullptr) {
+        int dev = -1;
+        if (cudaGetDevice(&dev) != cudaSuccess || dev < 0 || dev >= MAX_DEVICES) {
+            cudaGetLastError();
+            return SQAP_ERR_CUDA;
+        }
+        std::lock_guard<std::mutex> lock(mutex_);
+        if (!done_[dev]) {
+            const sqap_status st = fn(&value_[dev]);
+            if (st != SQAP_OK) return st;
+            done_[dev] = true;
+        }
+        if (out) *out = &value_[dev];
+        return SQAP_OK;
+    }
+
+private:
+    std::mutex mutex_;
+    bool done_[MAX_DEVICES] = {};
+    T value_[MAX_DEVICES] = {};
+};
+
+// Raises a kernel's dynamic shared-memory limit on the current device (for PerDevice<int>::run).
+template <typename K>
+inline sqap_status set_max_dynamic_smem(K kernel, int bytes) {
+    const cudaError_t e = cudaFuncSetAttribute(kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, bytes);
+    if (e != cudaSuccess) {
+        note_cuda_error(e);
+        return SQAP_ERR_CUDA;
+    }
+    return SQAP_OK;
+}
+
 inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 15u) == 0; }
 
 // Programmatic dependent launch, used along the short kernel chains of a decode step (quantizer -> weight
@@ -26,6 +81,11 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // whatever does not depend on that kernel (the streamers: fetch their first weights) and then calls pdl_wait(),
 // which returns once the earlier kernel has completed and its writes are visible. The earlier kernel calls
 // pdl_launch_dependents() as soon as it is running. Both calls do nothing in a kernel launched the plain way.
+// THE RULE every kernel launched through launch_dependent() obeys: before its pdl_wait() it writes NO global
+// memory and reads nothing that another kernel of the stream may write (in practice: packed weights and weight
+// scales only, which are immutable after packing). Since these kernels release their dependents before their own
+// wait, up to three kernels of a chain can be resident at once; the rule is what keeps the workspace (expanded
+// codes, row sums, scales), which consecutive calls rewrite, and the activations free of races.
 constexpr int PDL_MAX_ROWS = 32;   // the quantizers launch this way up to here (the row counts of decode steps)
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }

@@ -389,13 +389,7 @@ __global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
 
 template <int CPL>
 static void launch_gemv1(const LinearArgs& a, cudaStream_t s) {
-    static int blocks = 0;
-    if (!blocks) {
-        int dev = 0, sms = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        blocks = (sms > 0 ? sms : 148) * 3;
-    }
+    const int blocks = sm_count() * 3;
     const int need = (a.N + 7) / 8;
     const int grid = need < blocks ? need : blocks;
     cudaError_t e;
@@ -433,7 +427,14 @@ static sqap_status check_linear_args(int M, const sqap_weights* w, const sqap_we
     if (flags & ~allowed_flags) return SQAP_ERR_INVALID;
     const uint32_t force = flags & SQAP_L_FORCE_MASK;
     if ((force & (force - 1)) != 0) return SQAP_ERR_INVALID;  // at most one forced kernel
-    if (w_up && (w_up->N != w->N || w_up->K != w->K || w_up->half != w->half)) return SQAP_ERR_INVALID;
+    if (w_up && (w_up->N != w->N || w_up->K != w->K || w_up->half != w->half || w_up->device != w->device))
+        return SQAP_ERR_INVALID;
+    int dev = -1;
+    if (cudaGetDevice(&dev) != cudaSuccess) {
+        cudaGetLastError();
+        return SQAP_ERR_CUDA;
+    }
+    if (dev != w->device) return SQAP_ERR_INVALID;   // the packed weights live on another device than the current one
     if (w_up && out_dtype == SQAP_I32) return SQAP_ERR_INVALID;
     if (ldo < w->N) return SQAP_ERR_INVALID;
     if (M == 0) return SQAP_OK;

@@ -265,13 +265,7 @@ __global__ void __launch_bounds__(MMA_WARPS * 32, 2) w4a4_mma_kernel(LinearArgs 
 
 template <int NG>
 void launch_ng(const LinearArgs& a, cudaStream_t s) {
-    static int resident = 0;    // CTAs that fit the device at two per SM
-    if (!resident) {
-        int dev = 0, sms = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&sms, cudaDevAttrMultiProcessorCount, dev);
-        resident = 2 * (sms > 0 ? sms : 148);
-    }
+    const int resident = 2 * sm_count();    // CTAs that fit the device at two per SM
     const int n_rb = (a.N + 15) / 16;
     const int grid = n_rb < resident ? n_rb : resident;
     cudaError_t e;

@@ -361,37 +361,37 @@ sqap_status launch_linear_tcgen05_pair(const LinearArgs& a, cudaStream_t s) {
     k.status = device_status_word();
     if (!k.status) return SQAP_ERR_CUDA;
 
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(w4a4_tc_pair_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        if (e != cudaSuccess) {
-            note_cuda_error(e);
-            return SQAP_ERR_CUDA;
-        }
-        attr_set = true;
-    }
-    // CTA pairs that can be resident at once: a pair needs both SMs of one TPC, so this can be fewer than half
-    // the SM count; a persistent grid larger than that would run its surplus pairs as a second wave.
-    static int max_pairs = 0;
-    if (!max_pairs) {
-        cudaLaunchConfig_t cfg = {};
-        cfg.gridDim = dim3(static_cast<unsigned>(sm_count() / 2 * 2));
-        cfg.blockDim = dim3(THREADS);
-        cfg.dynamicSmemBytes = SMEM_BYTES;
-        cudaLaunchAttribute attr;
-        attr.id = cudaLaunchAttributeClusterDimension;
-        attr.val.clusterDim.x = 2;
-        attr.val.clusterDim.y = 1;
-        attr.val.clusterDim.z = 1;
-        cfg.attrs = &attr;
-        cfg.numAttrs = 1;
-        int n = 0;
-        if (cudaOccupancyMaxActiveClusters(&n, w4a4_tc_pair_kernel, &cfg) != cudaSuccess || n <= 0) {
-            cudaGetLastError();
-            n = sm_count() / 2;
-        }
-        max_pairs = n;
-    }
+    // Once per device: the shared-memory limit, and the number of CTA pairs that can be resident at once. A pair
+    // needs both SMs of one TPC, so this can be fewer than half the SM count; a persistent grid larger than that
+    // would run its surplus pairs as a second wave.
+    static PerDevice<int> setup;
+    const int* max_pairs_p = nullptr;
+    const sqap_status st = setup.run(
+        [](int* pairs) {
+            const sqap_status s0 = set_max_dynamic_smem(w4a4_tc_pair_kernel, SMEM_BYTES);
+            if (s0 != SQAP_OK) return s0;
+            cudaLaunchConfig_t cfg = {};
+            cfg.gridDim = dim3(static_cast<unsigned>(sm_count() / 2 * 2));
+            cfg.blockDim = dim3(THREADS);
+            cfg.dynamicSmemBytes = SMEM_BYTES;
+            cudaLaunchAttribute attr;
+            attr.id = cudaLaunchAttributeClusterDimension;
+            attr.val.clusterDim.x = 2;
+            attr.val.clusterDim.y = 1;
+            attr.val.clusterDim.z = 1;
+            cfg.attrs = &attr;
+            cfg.numAttrs = 1;
+            int n = 0;
+            if (cudaOccupancyMaxActiveClusters(&n, w4a4_tc_pair_kernel, &cfg) != cudaSuccess || n <= 0) {
+                cudaGetLastError();
+                n = sm_count() / 2;
+            }
+            *pairs = n;
+            return SQAP_OK;
+        },
+        &max_pairs_p);
+    if (st != SQAP_OK) return st;
+    const int max_pairs = *max_pairs_p;
     choose_token_tiles(a.M, k.n_tiles, max_pairs, BN_MAX, 128, &k.m_tiles, &k.BN);
     CUtensorMap tm_w, tm_u, tm_x;
     const uint32_t w_box_rows = k.swiglu ? BM / 2 : BM;

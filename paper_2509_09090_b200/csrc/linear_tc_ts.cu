@@ -372,15 +372,9 @@ sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s) {
         return SQAP_ERR_CUDA;
     if (!make_map(&tm_x, a.x8, a.M, a.K, k.BN, BKH, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
 
-    static bool attr_set = false;
-    if (!attr_set) {
-        cudaError_t e = cudaFuncSetAttribute(w4a4_tc_ts_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize, SMEM_BYTES);
-        if (e != cudaSuccess) {
-            note_cuda_error(e);
-            return SQAP_ERR_CUDA;
-        }
-        attr_set = true;
-    }
+    static PerDevice<int> setup;
+    const sqap_status st = setup.run([](int*) { return set_max_dynamic_smem(w4a4_tc_ts_kernel, SMEM_BYTES); });
+    if (st != SQAP_OK) return st;
     const int tiles = k.m_tiles * k.n_tiles;
     const int grid = tiles < sm_count() ? tiles : sm_count();
     w4a4_tc_ts_kernel<<<grid, THREADS, SMEM_BYTES, s>>>(tm_w, tm_u, tm_x, k);

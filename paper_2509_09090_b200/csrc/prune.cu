@@ -81,7 +81,10 @@ __global__ void __launch_bounds__(512) prune_select_kernel(sqap_prune_params p, 
     if (warp == 0 && m_fps > 0) {
         uint32_t key[CAND];
         int tu[CAND], tv[CAND];
-        const uint32_t inv_w = 0xFFFFFFFFu / static_cast<uint32_t>(p.grid_w) + 1u;   // j / grid_w = umulhi(j, inv_w), j < 2^16
+        // j / grid_w = umulhi(j, inv_w) for j < 2^16 and 2 <= grid_w; a one-token-wide grid (where the 32-bit
+        // reciprocal would wrap to 0) has t_v = j, t_u = 0 directly
+        const bool one_wide = p.grid_w == 1;
+        const uint32_t inv_w = one_wide ? 0u : 0xFFFFFFFFu / static_cast<uint32_t>(p.grid_w) + 1u;
 #pragma unroll
         for (int i = 0; i < CAND; ++i) {
             const int j = lane + 32 * i;
@@ -97,7 +100,7 @@ __global__ void __launch_bounds__(512) prune_select_kernel(sqap_prune_params p, 
             best = __reduce_max_sync(0xffffffffu, best);
             if ((best >> 10) == 0) break;  // remainder exhausted
             const int pj = 1023 - static_cast<int>(best & 1023u);
-            const int pv = static_cast<int>(__umulhi(static_cast<uint32_t>(pj), inv_w));
+            const int pv = one_wide ? pj : static_cast<int>(__umulhi(static_cast<uint32_t>(pj), inv_w));
             const int pu = pj - pv * p.grid_w;
             if ((pj & 31) == lane) keep[pj] = 2;
 #pragma unroll

@@ -534,26 +534,17 @@ __global__ void __launch_bounds__(1024) tensor_max_kernel(float* __restrict__ sc
     for (int i = threadIdx.x; i < M; i += blockDim.x) scales[i] = m;
 }
 
-static int num_sms() {
-    static int n = 0;
-    if (!n) {
-        int dev = 0;
-        cudaGetDevice(&dev);
-        cudaDeviceGetAttribute(&n, cudaDevAttrMultiProcessorCount, dev);
-        if (n <= 0) n = 148;
-    }
-    return n;
-}
-
 template <int E, int SINK>
 static void launch_rotate(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, const QuantOut& o,
                           cudaStream_t s) {
     const int T = K / E;
     const float norm = static_cast<float>(1.0 / sqrt(static_cast<double>(K)));
     const size_t smem = (32 + (T > 32 ? static_cast<size_t>(K) : 0)) * sizeof(float);
-    if (smem > 48 * 1024)
-        cudaFuncSetAttribute(quantize_rows_rotate_kernel<E, SINK>, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                             static_cast<int>(smem));
+    if (smem > 48 * 1024) {
+        static PerDevice<int> setup;   // one per kernel instantiation; the limit covers the longest supported row
+        if (setup.run([](int*) { return set_max_dynamic_smem(quantize_rows_rotate_kernel<E, SINK>, (32 + 16384) * 4); }) != SQAP_OK)
+            return;
+    }
     if (M <= PDL_MAX_ROWS) {
         const cudaError_t e = launch_dependent(quantize_rows_rotate_kernel<E, SINK>, dim3(M), dim3(T), smem, s, x, K, ldx, row_index, norm, o);
         if (e != cudaSuccess) note_cuda_error(e);
@@ -567,18 +558,11 @@ static sqap_status launch_quantize(const __half* x, int M, int K, int64_t ldx, c
                                    const QuantOut& o, cudaStream_t s) {
     if (rotate) {
         if (K == R4K) {
-            static bool attr_set = false;  // per process; the attribute is per function and device-independent here
-            if (!attr_set) {
-                cudaError_t e = cudaFuncSetAttribute(quantize_rotate4096_kernel<SINK>,
-                                                     cudaFuncAttributeMaxDynamicSharedMemorySize, R4K_SMEM);
-                if (e != cudaSuccess) {
-                    note_cuda_error(e);
-                    return SQAP_ERR_CUDA;
-                }
-                attr_set = true;
-            }
+            static PerDevice<int> setup;
+            const sqap_status st = setup.run([](int*) { return set_max_dynamic_smem(quantize_rotate4096_kernel<SINK>, R4K_SMEM); });
+            if (st != SQAP_OK) return st;
             int ctas = (M + R4K_ROWS - 1) / R4K_ROWS;
-            const int resident = 2 * num_sms();
+            const int resident = 2 * sm_count();
             if (ctas > resident) ctas = resident;
             if (M <= PDL_MAX_ROWS) {
                 const cudaError_t e = launch_dependent(quantize_rotate4096_kernel<SINK>, dim3(ctas), dim3(R4K_THREADS), R4K_SMEM, s,

@@ -126,7 +126,8 @@ def within_tolerance(got_bits: np.ndarray, ref_bits: np.ndarray, bf16: bool = Fa
     if bf16:
         g = (got_bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
         r = (ref_bits.astype(np.uint32) << 16).view(np.float32).astype(np.float64)
-        ulp = np.maximum(np.abs(r), 2.0 ** -126) * 2.0 ** -7
+        # one unit in the last place of bf16 (8 significant bits) at ref: 2^(floor(log2 |ref|) - 7)
+        ulp = np.exp2(np.floor(np.log2(np.maximum(np.abs(r), 2.0 ** -126))) - 7.0)
     else:
         g = got_bits.view(np.float16).astype(np.float64)
         r = ref_bits.view(np.float16).astype(np.float64)

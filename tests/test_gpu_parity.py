@@ -440,6 +440,66 @@ def test_linear_rejects_bad_arguments():
     w2.close()
 
 
+def test_decode_chain_back_to_back_on_one_workspace():
+    """A decode layer issued eagerly with no host synchronisation in between, every call on the same workspace, as a
+    layer runs it: quantize+linear with the row quantized inside the streamer, two more weight matrices on the
+    expanded codes it left (SQAP_L_REUSE_EXPANDED), the next fused call overwriting the workspace, a rotated call
+    (separate quantizer kernel launched as a programmatic dependent), twice around. Kernels of such a chain may
+    overlap their predecessor up to their dependency wait; every output must still equal the oracle's."""
+    K, N = 4096, 264
+    x = wl.activations(33, 1, 3, K, 41, 30.0)
+    ws_ = [(wl.weight_codes(33, 10 + i, N, K), wl.weight_scales(33, 10 + i, N, mult=0.25)) for i in range(4)]
+    w = [G.pack(c, s) for c, s in ws_]
+    xd = G.to_dev(x)
+    nb = B.sqap_quantize_linear_workspace_bytes(1, N, K)
+    wsp = torch.empty(nb, dtype=torch.uint8, device="cuda")
+    sc_ptr = wsp.data_ptr() + B.sqap_workspace_bytes(1, N, K)
+    outs = torch.full((2, 6, N), 0x7B7B, dtype=torch.int16, device="cuda")
+    dummy = torch.zeros(16, dtype=torch.uint8, device="cuda")
+    row = lambda r: xd.data_ptr() + 2 * K * r
+    for rep in range(2):
+        o = outs[rep]
+        B.sqap_quantize_linear(row(0), 1, K, None, 0, w[0], None, o[0], N, B.SQAP_FP16, 0, wsp, nb)
+        B.sqap_w4a4_linear(dummy, sc_ptr, 1, w[1], None, o[1], N, B.SQAP_FP16, B.SQAP_L_REUSE_EXPANDED, wsp, nb)
+        B.sqap_w4a4_linear(dummy, sc_ptr, 1, w[2], w[3], o[2], N, B.SQAP_FP16, B.SQAP_L_REUSE_EXPANDED, wsp, nb)
+        B.sqap_quantize_linear(row(1), 1, K, None, 0, w[2], w[3], o[3], N, B.SQAP_FP16, 0, wsp, nb)
+        B.sqap_quantize_linear(row(2), 1, K, None, B.SQAP_Q_ROTATE, w[1], None, o[4], N, B.SQAP_FP16, 0, wsp, nb)
+        B.sqap_w4a4_linear(dummy, sc_ptr, 1, w[0], None, o[5], N, B.SQAP_FP16, B.SQAP_L_REUSE_EXPANDED, wsp, nb)
+    torch.cuda.synchronize()
+    assert B.sqap_device_status() == B.SQAP_OK
+    got = outs.cpu().numpy().view(np.uint16)
+
+    def ref(r, rotate, g, u=None):
+        _, s, codes = oracle.quantize_act(bits(x[r:r + 1]), rotate=rotate)
+        acc = oracle.gemm_i32(codes, ws_[g][0])
+        if u is None:
+            return oracle.epilogue(acc, s, bits(ws_[g][1]))
+        return oracle.epilogue_swiglu(acc, oracle.gemm_i32(codes, ws_[u][0]), s, bits(ws_[g][1]), bits(ws_[u][1]))
+
+    want = [ref(0, False, 0), ref(0, False, 1), ref(0, False, 2, 3), ref(1, False, 2, 3), ref(2, True, 1), ref(2, True, 0)]
+    for rep in range(2):
+        for i, r in enumerate(want):
+            assert G.within_tolerance(got[rep, i][None], r).all(), (rep, i)
+    for h in w:
+        h.close()
+
+
+def test_bounded_wait_runs_out_and_reports_timeout():
+    """The failure-detection path: a wait that nothing satisfies gives up after its limit, the status word reports
+    SQAP_ERR_TIMEOUT exactly once, and the device keeps working (a linear right after matches the oracle)."""
+    assert B.sqap_device_status() == B.SQAP_OK
+    L = B.lib()
+    assert L.sqap_selftest_bounded_wait(10, None) == B.SQAP_ERR_INVALID
+    assert L.sqap_selftest_bounded_wait(10 ** 10, None) == B.SQAP_ERR_INVALID
+    B.sqap_selftest_bounded_wait(2_000_000)          # about a millisecond
+    assert B.sqap_device_status() == B.SQAP_ERR_TIMEOUT
+    assert B.sqap_device_status() == B.SQAP_OK
+    M, N, K = 150, 256, 512
+    x = wl.activations(34, 1, M, K, 5, 20.0)
+    check_linear(x, wl.weight_codes(34, 2, N, K), wl.weight_scales(34, 2, N),
+                 flags_list=[B.SQAP_L_FORCE_TCGEN05_TS, B.SQAP_L_FORCE_TCGEN05_PAIR])
+
+
 # ------------------------------------------------------------------ pruning
 
 def check_prune(params, scores, centers=None, x=None, out_rows=0):
@@ -493,6 +553,18 @@ def test_prune_ties_large_grid_and_ragged_rows():
     p = wl.prune_params(2, 10, 0, 0, 0, 0, 0, 0, 0)
     kept, nk, _ = G.prune(p, np.zeros((2, 1), np.float32))
     assert (nk == 10).all() and (kept == np.arange(10)).all()
+
+
+@pytest.mark.parametrize("grid_w,grid_h", [(1, 40), (40, 1), (1, 1), (2, 33), (1, 1024)])
+def test_prune_fps_on_one_token_wide_and_high_grids(grid_w, grid_h):
+    """Grids that are a single column or a single row of tokens, with farthest-point sampling active (and a ring,
+    and some top-k): the picked token's coordinates must come out right when grid_w = 1."""
+    nv = grid_w * grid_h
+    rng = np.random.default_rng(grid_w * 1000 + grid_h)
+    s = rng.integers(0, 4, (2, nv)).astype(np.float32)
+    for k_attn, keep, radius in [(0, nv // 2 + 1, -1), (min(3, nv), min(nv, 17), 1), (0, nv, -1)]:
+        p = wl.prune_params(2, nv + 9, 4, nv, grid_w, grid_h, 0, k_attn, keep, ring_radius=radius)
+        check_prune(p, s, np.array([[0, grid_h // 2], [grid_w - 1, 0]], np.int32))
 
 
 def test_prune_fps_worked_example():
@@ -606,9 +678,26 @@ def test_config3_decode_step_gemv():
     check_linear(h, lw["down_codes"], lw["down_scales"], flags_list=[0])
 
 
-@pytest.mark.parametrize("keep", [64, 192, 256])
+def _check_sampled(acc, out, codes, so, wc, ws, rng, M, N):
+    """Whole sampled rows and columns and 512 single entries of a full-size GEMM against the oracle; returns the
+    sampled row numbers and their oracle accumulators."""
+    rows = np.unique(np.concatenate([[0, M - 1, 255, 256], rng.integers(0, M, 4)]))
+    ref_rows = oracle.gemm_i32(codes[rows], wc)
+    assert np.array_equal(acc[rows], ref_rows)
+    assert G.within_tolerance(out[rows], oracle.epilogue(ref_rows, so[rows], bits(ws))).all()
+    cols = np.unique(np.concatenate([[0, N - 1, 127, 128], rng.integers(0, N, 4)]))
+    ref_cols = oracle.gemm_i32(codes, wc[cols])
+    assert np.array_equal(acc[:, cols], ref_cols)
+    for _ in range(512):
+        m, n = int(rng.integers(0, M)), int(rng.integers(0, N))
+        assert acc[m, n] == oracle.dot_i32(codes[m], wc[n])
+    return rows, ref_rows
+
+
+@pytest.mark.parametrize("keep", [64, 128, 192, 256])
 def test_config4_batched_sampled(keep):
-    """Full-size GEMMs (M up to 4608): accumulators checked on sampled entries and on whole sampled rows."""
+    """Full-size GEMMs (M = 1536, 2560, 3584, 4608; every shape of the layer, the down projection with its 11008
+    codes per row included): accumulators checked on sampled entries and on whole sampled rows and columns."""
     Bn = 16
     inp = wl.config4_inputs()
     wts = wl.config4_weights()
@@ -630,16 +719,7 @@ def test_config4_batched_sampled(keep):
         w = G.pack(wc, ws)
         acc = G.linear(pg, sg, w, out_dtype=B.SQAP_I32)
         out = G.linear(pg, sg, w)
-        rows = np.unique(np.concatenate([[0, M - 1, 255, 256], rng.integers(0, M, 4)]))
-        ref_rows = oracle.gemm_i32(codes[rows], wc)
-        assert np.array_equal(acc[rows], ref_rows)
-        assert G.within_tolerance(out[rows], oracle.epilogue(ref_rows, so[rows], bits(ws))).all()
-        cols = np.unique(np.concatenate([[0, N - 1, 127, 128], rng.integers(0, N, 4)]))
-        ref_cols = oracle.gemm_i32(codes, wc[cols])
-        assert np.array_equal(acc[:, cols], ref_cols)
-        for _ in range(512):
-            m, n = int(rng.integers(0, M)), int(rng.integers(0, N))
-            assert acc[m, n] == oracle.dot_i32(codes[m], wc[n])
+        rows, ref_rows = _check_sampled(acc, out, codes, so, wc, ws, rng, M, N)
         if name == "gate":
             wu = G.pack(wts["up_codes"], wts["up_scales"])
             hs = G.linear(pg, sg, w, w_up=wu)
@@ -648,3 +728,16 @@ def test_config4_batched_sampled(keep):
             assert G.within_tolerance(hs[rows], ref_h).all()
             wu.close()
         w.close()
+    # the down projection: rows of 11008 codes (43 pipeline stages of 256), fed by a stand-in for the gated MLP output
+    del codes, po, pg
+    xh = wl.activations(4, 900 + keep, M, wl.FFN, 110, 30.0)
+    po, so, codes = oracle.quantize_act(bits(xh))
+    pg, sg = G.quantize(xh)
+    assert np.array_equal(pg, po) and np.array_equal(sg, so)
+    wc, ws = wts["down_codes"], wts["down_scales"]
+    w = G.pack(wc, ws)
+    acc = G.linear(pg, sg, w, out_dtype=B.SQAP_I32)
+    out = G.linear(pg, sg, w)
+    _check_sampled(acc, out, codes, so, wc, ws, rng, M, wl.HIDDEN)
+    assert np.array_equal(G.quantize_linear(xh, w), out)       # the one-call route the layer uses
+    w.close()

@@ -13,6 +13,7 @@ Collected last on purpose: if it fails under `-x`, every other test has already 
 import numpy as np
 import pytest
 
+import oracle
 from paper_2509_09090_b200 import workloads as wl
 
 pytestmark = pytest.mark.gpu
@@ -57,6 +58,19 @@ def test_static_scratch_linear_matches_workspace_linear_twice_in_a_row():
         # 2e-3) is met with room to spare — the bits are identical
         assert np.array_equal(first, want)
         assert np.array_equal(second, want)
+        # and against the CPU oracle, so that a defect shared by both entry points cannot pass: exact integers,
+        # fp16 within max(1 ulp, 2e-3 relative)
+        _, so, codes = oracle.quantize_act(np.ascontiguousarray(x).view(np.uint16))
+        wc, sw = wl.weight_codes(77, N + K, N, K), wl.weight_scales(77, N + K, N, mult=0.5).view(np.uint16)
+        acc = oracle.gemm_i32(codes, wc)
+        if kind == "i32":
+            assert np.array_equal(second, acc)
+        elif fused:
+            acc_u = oracle.gemm_i32(codes, wl.weight_codes(77, N + K + 1, N, K))
+            su = wl.weight_scales(77, N + K + 1, N, mult=0.5).view(np.uint16)
+            assert G.within_tolerance(second, oracle.epilogue_swiglu(acc, acc_u, so, sw, su)).all()
+        else:
+            assert G.within_tolerance(second, oracle.epilogue(acc, so, sw)).all()
         w.close()
         if wu:
             wu.close()
