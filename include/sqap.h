@@ -60,9 +60,13 @@ typedef enum {
                                        (needs K % 128 == 0) */
 #define SQAP_L_FORCE_TCGEN05_PAIR 32u /* the same on CTA pairs (tcgen05 cta_group::2) */
 #define SQAP_L_FORCE_MMA 64u /* the register-MMA weight streamer for a handful of rows (M <= 32, K % 128 == 0) */
+#define SQAP_L_FORCE_TCGEN05_SPLITK 128u /* the tcgen05 kernel that splits K over the CTAs of a cluster (needs
+                                            K % 128 == 0); SQAP_L_KSPLIT(n), n = 1..4, also fixes the cluster size */
+#define SQAP_L_KSPLIT(n) ((uint32_t)(n) << 8)
+#define SQAP_L_KSPLIT_MASK 0x700u
 #define SQAP_L_FORCE_MASK                                                                                          \
     (SQAP_L_FORCE_SIMT | SQAP_L_FORCE_TCGEN05 | SQAP_L_FORCE_GEMV | SQAP_L_FORCE_TCGEN05_TS | SQAP_L_FORCE_TCGEN05_PAIR | \
-     SQAP_L_FORCE_MMA)
+     SQAP_L_FORCE_MMA | SQAP_L_FORCE_TCGEN05_SPLITK)
 #define SQAP_L_REUSE_EXPANDED 8u /* the workspace still holds the expanded form of these same M x K activations
                                     from the previous call that used it (one activation feeding several weight
                                     matrices): skip the expand pass */

@@ -20,6 +20,11 @@ SQAP_Q_PER_TENSOR = 2
 SQAP_W_ROTATED = 1
 SQAP_L_FORCE_SIMT, SQAP_L_FORCE_TCGEN05, SQAP_L_FORCE_GEMV, SQAP_L_REUSE_EXPANDED, SQAP_L_FORCE_TCGEN05_TS, SQAP_L_FORCE_TCGEN05_PAIR = 1, 2, 4, 8, 16, 32
 SQAP_L_FORCE_MMA = 64
+SQAP_L_FORCE_TCGEN05_SPLITK = 128
+
+
+def SQAP_L_KSPLIT(n: int) -> int:
+    return n << 8
 
 EXPORTS = ("sqap_pack_weights", "sqap_quantize_weights", "sqap_free_weights", "sqap_weights_info", "sqap_unpack_weights",
            "sqap_quantize_act", "sqap_quantize_act_ex", "sqap_workspace_bytes", "sqap_w4a4_linear", "sqap_w4a4_linear_static",

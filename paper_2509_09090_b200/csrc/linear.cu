@@ -417,14 +417,15 @@ static size_t round256(size_t v) { return (v + 255) / 256 * 256; }
 
 namespace sqap {
 
-enum LinearPath { PATH_SIMT, PATH_TC, PATH_TC_TS, PATH_TC_PAIR, PATH_GEMV, PATH_MMA };
+enum LinearPath { PATH_SIMT, PATH_TC, PATH_TC_TS, PATH_TC_PAIR, PATH_TC_SPLITK, PATH_GEMV, PATH_MMA };
 
 // Argument rules shared by the entry points that run a linear (everything except the activation side).
 static sqap_status check_linear_args(int M, const sqap_weights* w, const sqap_weights* w_up, const void* out,
                                      int64_t ldo, int out_dtype, uint32_t flags, uint32_t allowed_flags) {
     if (M < 0 || !w) return SQAP_ERR_INVALID;
     if (out_dtype != SQAP_FP16 && out_dtype != SQAP_BF16 && out_dtype != SQAP_I32) return SQAP_ERR_INVALID;
-    if (flags & ~allowed_flags) return SQAP_ERR_INVALID;
+    if (flags & ~(allowed_flags | SQAP_L_KSPLIT_MASK)) return SQAP_ERR_INVALID;
+    if ((flags & SQAP_L_KSPLIT_MASK) && !(flags & SQAP_L_FORCE_TCGEN05_SPLITK)) return SQAP_ERR_INVALID;
     const uint32_t force = flags & SQAP_L_FORCE_MASK;
     if ((force & (force - 1)) != 0) return SQAP_ERR_INVALID;  // at most one forced kernel
     if (w_up && (w_up->N != w->N || w_up->K != w->K || w_up->half != w->half || w_up->device != w->device))
@@ -481,6 +482,9 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
     } else if (flags & SQAP_L_FORCE_TCGEN05_PAIR) {
         if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
         *path = PATH_TC_PAIR;
+    } else if (flags & SQAP_L_FORCE_TCGEN05_SPLITK) {
+        if (!tcgen05_supports(a)) return SQAP_ERR_UNSUPPORTED;
+        *path = PATH_TC_SPLITK;
     } else if (flags & SQAP_L_FORCE_MMA) {
         if (!mma_stream_supports(a)) return SQAP_ERR_UNSUPPORTED;
         *path = PATH_MMA;
@@ -498,13 +502,15 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
         const bool gemv = !stream && a.M <= 8 && (!tc_ok || a.M <= 2 || (a.M <= 4 && w_tiles < 64));
         // CTA pairs fetch each token once per 256 weight rows: ahead from ~144 tokens on when there are enough pairs
         const bool pairs = a.M >= 512 || (a.M >= 144 && w_tiles >= 64);
-        *path = stream ? PATH_MMA : gemv ? PATH_GEMV : (tc_ok ? (pairs ? PATH_TC_PAIR : PATH_TC_TS) : PATH_SIMT);
+        *path = stream ? PATH_MMA : gemv ? PATH_GEMV : (tc_ok ? (pairs ? PATH_TC_PAIR : PATH_TC_SPLITK) : PATH_SIMT);
     }
     return SQAP_OK;
 }
 
-static sqap_status run_gemm(const LinearArgs& a, LinearPath path, cudaStream_t s) {
+static sqap_status run_gemm(const LinearArgs& a, LinearPath path, uint32_t flags, cudaStream_t s) {
     if (path == PATH_TC) return launch_linear_tcgen05(a, s);
+    if (path == PATH_TC_SPLITK)
+        return launch_linear_tcgen05_splitk(a, static_cast<int>((flags & SQAP_L_KSPLIT_MASK) >> 8), s);
     if (path == PATH_TC_TS) return launch_linear_tcgen05_ts(a, s);
     if (path == PATH_TC_PAIR) return launch_linear_tcgen05_pair(a, s);
     if (path == PATH_MMA) return launch_linear_mma_stream(a, s);
@@ -561,7 +567,7 @@ sqap_status sqap_w4a4_linear(const uint8_t* q_packed, const float* act_scales, i
         st = check_launch();
         if (st != SQAP_OK) return st;
     }
-    return run_gemm(a, path, s);
+    return run_gemm(a, path, flags, s);
 }
 
 size_t sqap_quantize_linear_workspace_bytes(int M, int N, int K) {
@@ -594,12 +600,12 @@ sqap_status sqap_quantize_linear(const void* x, int M, int64_t ldx, const int32_
         a.fuse_x = static_cast<const __half*>(x);
         a.fuse_ldx = ldx;
         a.fuse_row_index = row_index;
-        return run_gemm(a, path, s);
+        return run_gemm(a, path, lflags, s);
     }
     st = quantize_expanded(static_cast<const __half*>(x), M, a.K, ldx, row_index, qflags, a.half,
                            const_cast<int8_t*>(a.x8), const_cast<int32_t*>(a.bias_sum), scales, s);
     if (st != SQAP_OK) return st;
-    return run_gemm(a, path, s);
+    return run_gemm(a, path, lflags, s);
 }
 
 }  // extern "C"

@@ -52,6 +52,10 @@ sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s);
 // The same on CTA pairs (linear_tc_pair.cu): the large-M kernel. Runs every shape the kernels above run.
 sqap_status launch_linear_tcgen05_pair(const LinearArgs& a, cudaStream_t s);
 
+// One cluster per tile with K split over its CTAs (linear_tc_splitk.cu): the kernel for a few dozen to a few
+// hundred tokens. Runs every shape the kernels above run. forced_split: 0 = choose, 1..4 = that cluster size.
+sqap_status launch_linear_tcgen05_splitk(const LinearArgs& a, int forced_split, cudaStream_t s);
+
 
 // Register-MMA weight streamer for a handful of tokens (linear_mma.cu): K % 128 == 0 and M <= MMA_STREAM_MAX_M.
 constexpr int MMA_STREAM_MAX_M = 32;

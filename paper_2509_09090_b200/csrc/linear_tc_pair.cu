@@ -40,7 +40,8 @@ constexpr int OFF_X = 0;
 constexpr int OFF_WP = OFF_X + S * 2 * XH_BYTES;
 constexpr int OFF_BAR = OFF_WP + S * 2 * WPH_BYTES;
 constexpr int OFF_TOK = OFF_BAR + 512;    // per-token epilogue constants, two tiles x BN_MAX x 8 bytes
-constexpr int SMEM_BYTES = OFF_TOK + 2 * BN_MAX * 8 + 1024;  // + slack for 1024-byte alignment
+constexpr int OFF_STAGE = OFF_TOK + 2 * BN_MAX * 8;   // staging of the coalesced epilogue (tc_common.cuh)
+constexpr int SMEM_BYTES = OFF_STAGE + EPI_STAGE_TOTAL + 1024;  // + slack for 1024-byte alignment
 constexpr int TMEM_A_COL = 2 * BN_MAX;    // columns [0,192) and [192,384): accumulators; from 384: weight tiles
 constexpr int A_COLS = BK / 4;            // 64 columns hold 256 int8 per lane
 constexpr int EPI_WARPS = 8;
@@ -314,12 +315,16 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
                 n_ok = n < a.N;
                 sw = n_ok ? __half2float(a.w_scales[n]) : 0.0f;
             }
+            // fp16 / bf16: through shared memory, 16 bytes per thread to global memory; raw int32 (checking): directly
+            const int hf = (warp - 6) >> 2, tid_half = static_cast<int>(threadIdx.x) - (6 + 4 * hf) * 32;
+            uint8_t* stage_half = sm + OFF_STAGE + hf * 2 * EPI_STAGE_BYTES;
             if (a.swiglu) {
-                if (a.out_dtype == SQAP_FP16) epilogue_tile_staged<SQAP_FP16, true, 16>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane, tok);
-                else epilogue_tile_staged<SQAP_BF16, true, 16>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane, tok);
+                const int ch = quad * 16 + (lane & 15);
+                if (a.out_dtype == SQAP_FP16) epilogue_tile_coalesced<SQAP_FP16, true>(a, taddr, m0, c_begin, c_end, n0 / 2, ch, sw, lane, tok, stage_half, tid_half, 2 + hf);
+                else epilogue_tile_coalesced<SQAP_BF16, true>(a, taddr, m0, c_begin, c_end, n0 / 2, ch, sw, lane, tok, stage_half, tid_half, 2 + hf);
             } else {
-                if (a.out_dtype == SQAP_FP16) epilogue_tile_staged<SQAP_FP16, false, 1>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane, tok);
-                else if (a.out_dtype == SQAP_BF16) epilogue_tile_staged<SQAP_BF16, false, 1>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane, tok);
+                if (a.out_dtype == SQAP_FP16) epilogue_tile_coalesced<SQAP_FP16, false>(a, taddr, m0, c_begin, c_end, n0, row, sw, lane, tok, stage_half, tid_half, 2 + hf);
+                else if (a.out_dtype == SQAP_BF16) epilogue_tile_coalesced<SQAP_BF16, false>(a, taddr, m0, c_begin, c_end, n0, row, sw, lane, tok, stage_half, tid_half, 2 + hf);
                 else epilogue_tile_staged<SQAP_I32, false, 1>(a, taddr, m0, c_begin, c_end, n, n_ok, sw, lane, tok);
             }
             tc_fence_before();

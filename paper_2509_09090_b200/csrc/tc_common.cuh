@@ -230,54 +230,148 @@ __device__ __forceinline__ bool bar_or(int id, int nthreads, bool pred) {
     return r != 0;
 }
 
-// The same epilogue with the per-token constants staged in shared memory: tok[c] = {128 * bias_sum, bits of the
-// activation scale} of token m0 + c ({0, 0} past M). All lanes of a warp need the same token's pair, so one
-// broadcast shared-memory load per two tokens replaces four warp shuffles; the shuffles of the routine above
-// share a pipe with the unpack warps' shared-memory loads and were measured to slow the main loop.
+// One 16-token chunk of an accumulator tile, raw sums in registers -> global memory. The thread owns one output
+// channel n (one tensor-memory lane; with SwiGLU the gate and up projections of a channel sit in lanes XCHG apart)
+// and 16 consecutive tokens, the first of which is token `m_first` of the matrix. t4 points at the staged
+// per-token constants of those tokens: {128 * bias_sum, bits of the activation scale} per token ({0, 0} past M),
+// two tokens per 16-byte shared-memory load (a broadcast: every lane of a warp needs the same pair).
 template <int OUT, bool SWIGLU, int XCHG>
-__device__ __forceinline__ void epilogue_tile_staged(const Args& a, uint32_t taddr, int m0, int c_begin, int c_end, int n,
-                                                     bool n_ok, float sw, int lane, const int2* tok) {
+__device__ __forceinline__ void epilogue_chunk(const Args& a, const uint32_t* v, int m_first, int n, bool n_ok, float sw,
+                                               int lane, const int4* t4) {
     constexpr int ESZ = OUT == SQAP_I32 ? 4 : 2;
     const bool odd = (lane & XCHG) != 0;   // SwiGLU: this lane holds the up projection, its partner (lane ^ XCHG) the gate
     const int64_t row_bytes = a.ldo * ESZ;
+    const int valid = a.M - m_first;  // tokens of this chunk that exist
+    uint8_t* optr = static_cast<uint8_t*>(a.out) + static_cast<int64_t>(m_first) * row_bytes + static_cast<int64_t>(n) * ESZ;
+#pragma unroll
+    for (int j = 0; j < 16; j += 2) {
+        const int4 t = t4[j >> 1];
+        const int t0 = (static_cast<int>(v[j]) - t.x) >> 4, t1 = (static_cast<int>(v[j + 1]) - t.z) >> 4;
+        const float y0 = __fmul_rn(__fmul_rn(static_cast<float>(t0), __int_as_float(t.y)), sw);
+        const float y1 = __fmul_rn(__fmul_rn(static_cast<float>(t1), __int_as_float(t.w)), sw);
+        if (SWIGLU) {
+            // the gate lane finishes token j (needs the up value of its partner), the up lane token j+1
+            const float got = __shfl_xor_sync(0xffffffffu, odd ? y0 : y1, XCHG);
+            const float h = odd ? silu_mul_fast(got, y1) : silu_mul_fast(y0, got);
+            const int jj = odd ? j + 1 : j;
+            if (n_ok && jj < valid) {
+                uint8_t* o = optr + jj * row_bytes;
+                if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(h);
+                else *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(h);
+            }
+        } else {
+            if (n_ok && j < valid) {
+                uint8_t* o = optr + j * row_bytes;
+                if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(y0);
+                else if (OUT == SQAP_BF16) *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(y0);
+                else *reinterpret_cast<int32_t*>(o) = t0;
+            }
+            if (n_ok && j + 1 < valid) {
+                uint8_t* o = optr + (j + 1) * row_bytes;
+                if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(y1);
+                else if (OUT == SQAP_BF16) *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(y1);
+                else *reinterpret_cast<int32_t*>(o) = t1;
+            }
+        }
+    }
+}
+
+// Part of one finished accumulator tile -> global memory, with the per-token constants staged in shared memory:
+// tok[c] = {128 * bias_sum, bits of the activation scale} of token m0 + c ({0, 0} past M). One broadcast
+// shared-memory load per two tokens; fetching them by warp shuffles instead (the routine above) was measured to
+// slow the main loop, because shuffles share a pipe with the unpack warps' shared-memory loads.
+template <int OUT, bool SWIGLU, int XCHG>
+__device__ __forceinline__ void epilogue_tile_staged(const Args& a, uint32_t taddr, int m0, int c_begin, int c_end, int n,
+                                                     bool n_ok, float sw, int lane, const int2* tok) {
     for (int c = c_begin; c < c_end; c += 16) {
         uint32_t v[16];
         tc_ld16(taddr + c, v);
         const int4* t4 = reinterpret_cast<const int4*>(tok + c);   // two tokens per 16-byte load
         tc_wait_ld();
-        const int valid = a.M - (m0 + c);  // tokens of this chunk that exist
-        uint8_t* optr = static_cast<uint8_t*>(a.out) + static_cast<int64_t>(m0 + c) * row_bytes + static_cast<int64_t>(n) * ESZ;
+        epilogue_chunk<OUT, SWIGLU, XCHG>(a, v, m0 + c, n, n_ok, sw, lane, t4);
+    }
+}
+
+// ---- epilogue with coalesced global stores (fp16 / bf16 outputs)
+// In tensor memory a thread owns one output channel and a row of tokens, while in the output matrix the channels of
+// one token are contiguous: stored straight from registers, a warp writes 64 bytes per instruction (32 channels x
+// 2 bytes of one token), and those narrow stores were measured to take about 100 cycles each per warp. Here the 128
+// threads that share a half of the tile's tokens (one warp per lane quadrant) first put each 16-token chunk into
+// shared memory as [token][channel], meet at a named barrier, and copy it out 16 bytes per thread, 512 contiguous
+// bytes per warp instruction. Two buffers per half take turns, so one barrier per chunk is enough: a thread can
+// only be two chunks ahead of the slowest after passing the barrier in between, which every thread reaches after
+// its own copy-out of the chunk before.
+constexpr int EPI_STAGE_BYTES = 16 * 128 * 2;                // one chunk: 16 tokens x up to 128 channels x 2 bytes
+constexpr int EPI_STAGE_TOTAL = 2 * 2 * EPI_STAGE_BYTES;     // two halves x two buffers
+
+__device__ __forceinline__ void bar_sync_named(int id, int nthreads) {
+    asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
+}
+
+// v: the raw sums of this thread's channel for 16 consecutive tokens starting at token m_first of the matrix.
+// ch: the thread's channel within the tile (plain: 0..127 = tensor-memory lane; SwiGLU: 0..63, gate and up of a
+// channel sit 16 lanes apart); n_tile0: first output channel of the tile; sw: this lane's weight scale.
+// stage: the buffer for this chunk; tid_half: 0..127 among the threads sharing it; bar_id: their named barrier.
+template <int OUT, bool SWIGLU>
+__device__ __forceinline__ void epilogue_chunk_coalesced(const Args& a, const uint32_t* v, int m_first, int n_tile0, int ch,
+                                                         float sw, int lane, const int4* t4, uint8_t* stage, int tid_half,
+                                                         int bar_id) {
+    static_assert(OUT == SQAP_FP16 || OUT == SQAP_BF16, "16-bit outputs only");
+    constexpr int ROWB = SWIGLU ? 128 : 256;   // bytes of one token's channels in the buffer
+    auto bits16 = [](float y) -> uint16_t {
+        return OUT == SQAP_FP16 ? __half_as_ushort(__float2half_rn(y)) : __bfloat16_as_ushort(__float2bfloat16_rn(y));
+    };
+    const bool odd = (lane & 16) != 0;         // SwiGLU: this lane holds the up projection, lane ^ 16 the gate
+    uint8_t* mine = stage + ch * 2;
 #pragma unroll
-        for (int j = 0; j < 16; j += 2) {
-            const int4 t = t4[j >> 1];
-            const int t0 = (static_cast<int>(v[j]) - t.x) >> 4, t1 = (static_cast<int>(v[j + 1]) - t.z) >> 4;
-            const float y0 = __fmul_rn(__fmul_rn(static_cast<float>(t0), __int_as_float(t.y)), sw);
-            const float y1 = __fmul_rn(__fmul_rn(static_cast<float>(t1), __int_as_float(t.w)), sw);
-            if (SWIGLU) {
-                // the gate lane finishes token j (needs the up value of its partner), the up lane token j+1
-                const float got = __shfl_xor_sync(0xffffffffu, odd ? y0 : y1, XCHG);
-                const float h = odd ? silu_mul_fast(got, y1) : silu_mul_fast(y0, got);
-                const int jj = odd ? j + 1 : j;
-                if (n_ok && jj < valid) {
-                    uint8_t* o = optr + jj * row_bytes;
-                    if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(h);
-                    else *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(h);
-                }
+    for (int j = 0; j < 16; j += 2) {
+        const int4 t = t4[j >> 1];
+        const int t0 = (static_cast<int>(v[j]) - t.x) >> 4, t1 = (static_cast<int>(v[j + 1]) - t.z) >> 4;
+        const float y0 = __fmul_rn(__fmul_rn(static_cast<float>(t0), __int_as_float(t.y)), sw);
+        const float y1 = __fmul_rn(__fmul_rn(static_cast<float>(t1), __int_as_float(t.w)), sw);
+        if (SWIGLU) {
+            // the gate lane finishes token j (needs the up value of its partner), the up lane token j+1
+            const float got = __shfl_xor_sync(0xffffffffu, odd ? y0 : y1, 16);
+            const float h = odd ? silu_mul_fast(got, y1) : silu_mul_fast(y0, got);
+            *reinterpret_cast<uint16_t*>(mine + (odd ? j + 1 : j) * ROWB) = bits16(h);
+        } else {
+            *reinterpret_cast<uint16_t*>(mine + j * ROWB) = bits16(y0);
+            *reinterpret_cast<uint16_t*>(mine + (j + 1) * ROWB) = bits16(y1);
+        }
+    }
+    bar_sync_named(bar_id, 128);
+    constexpr int PPR = ROWB / 16;             // 16-byte pieces (8 channels) per token
+#pragma unroll
+    for (int p = tid_half; p < 16 * PPR; p += 128) {
+        const int token = p / PPR, piece = p % PPR;
+        const int m = m_first + token, n = n_tile0 + piece * 8;
+        if (m < a.M && n < a.N) {
+            const uint8_t* src = stage + token * ROWB + piece * 16;
+            uint8_t* dst = static_cast<uint8_t*>(a.out) + (static_cast<int64_t>(m) * a.ldo + n) * 2;
+            if (n + 8 <= a.N) {
+                *reinterpret_cast<uint4*>(dst) = *reinterpret_cast<const uint4*>(src);
             } else {
-                if (n_ok && j < valid) {
-                    uint8_t* o = optr + j * row_bytes;
-                    if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(y0);
-                    else if (OUT == SQAP_BF16) *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(y0);
-                    else *reinterpret_cast<int32_t*>(o) = t0;
-                }
-                if (n_ok && j + 1 < valid) {
-                    uint8_t* o = optr + (j + 1) * row_bytes;
-                    if (OUT == SQAP_FP16) *reinterpret_cast<__half*>(o) = __float2half_rn(y1);
-                    else if (OUT == SQAP_BF16) *reinterpret_cast<__nv_bfloat16*>(o) = __float2bfloat16_rn(y1);
-                    else *reinterpret_cast<int32_t*>(o) = t1;
-                }
+                for (int e = 0; e < a.N - n; ++e)
+                    reinterpret_cast<uint16_t*>(dst)[e] = reinterpret_cast<const uint16_t*>(src)[e];
             }
         }
+    }
+}
+
+// Tokens [c_begin, c_end) of a finished accumulator tile through the routine above. stage_half: this half's two
+// buffers (2 * EPI_STAGE_BYTES); tok as in epilogue_tile_staged.
+template <int OUT, bool SWIGLU>
+__device__ __forceinline__ void epilogue_tile_coalesced(const Args& a, uint32_t taddr, int m0, int c_begin, int c_end,
+                                                        int n_tile0, int ch, float sw, int lane, const int2* tok,
+                                                        uint8_t* stage_half, int tid_half, int bar_id) {
+    int flip = 0;
+    for (int c = c_begin; c < c_end; c += 16, flip ^= 1) {
+        uint32_t v[16];
+        tc_ld16(taddr + c, v);
+        const int4* t4 = reinterpret_cast<const int4*>(tok + c);   // two tokens per 16-byte load
+        tc_wait_ld();
+        epilogue_chunk_coalesced<OUT, SWIGLU>(a, v, m0 + c, n_tile0, ch, sw, lane, t4, stage_half + flip * EPI_STAGE_BYTES,
+                                              tid_half, bar_id);
     }
 }
 

@@ -278,8 +278,9 @@ def test_linear_tcgen05_forced(M, N, K, swiglu):
     x = wl.activations(25, M + K, M, K, max(1, K // 100), 20.0)
     g = (wl.weight_codes(25, N + K, N, K), wl.weight_scales(25, N + K, N, mult=0.5))
     u = (wl.weight_codes(25, N + K + 1, N, K), wl.weight_scales(25, N + K + 1, N, mult=0.5)) if swiglu else None
-    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS, B.SQAP_L_FORCE_TCGEN05_PAIR])
-    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS, B.SQAP_L_FORCE_TCGEN05_PAIR], bf16=True)
+    kernels = [B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS, B.SQAP_L_FORCE_TCGEN05_PAIR, B.SQAP_L_FORCE_TCGEN05_SPLITK]
+    check_linear(x, g[0], g[1], up=u, flags_list=kernels)
+    check_linear(x, g[0], g[1], up=u, flags_list=kernels, bf16=True)
 
 
 @pytest.mark.parametrize("M,N,K,swiglu", [(1300, 3500, 384, False), (1000, 2368, 256, True)])
@@ -289,7 +290,45 @@ def test_linear_tcgen05_many_tiles(M, N, K, swiglu):
     x = wl.activations(26, M + K, M, K, max(1, K // 100), 20.0)
     g = (wl.weight_codes(26, N + K, N, K), wl.weight_scales(26, N + K, N, mult=0.5))
     u = (wl.weight_codes(26, N + K + 1, N, K), wl.weight_scales(26, N + K + 1, N, mult=0.5)) if swiglu else None
-    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS, B.SQAP_L_FORCE_TCGEN05_PAIR])
+    check_linear(x, g[0], g[1], up=u, flags_list=[B.SQAP_L_FORCE_TCGEN05, B.SQAP_L_FORCE_TCGEN05_TS, B.SQAP_L_FORCE_TCGEN05_PAIR,
+                                                  B.SQAP_L_FORCE_TCGEN05_SPLITK])
+
+
+@pytest.mark.parametrize("M,N,K,swiglu,split", [
+    (160, 384, 4096, False, 4), (160, 264, 11008, False, 4), (288, 384, 4096, False, 2), (150, 320, 768, True, 3),
+    (17, 130, 1024, False, 4), (192, 256, 1280, True, 2), (100, 200, 2048, False, 3), (511, 136, 512, False, 2),
+    (33, 72, 256, False, 1), (160, 1024, 4096, True, 3), (176, 640, 2816, False, 0), (64, 4096, 1024, False, 0)])
+def test_linear_cluster_split_k(M, N, K, swiglu, split):
+    """The kernel that splits K over the CTAs of a cluster and adds the partial accumulators through distributed
+    shared memory: every cluster size, stage counts that do not divide evenly among the CTAs (43 over 4, 5 over 2,
+    8 over 3), one stage per CTA, two token tiles, chunk counts that leave some CTAs of the cluster one chunk
+    short, partial weight tiles, the fused gate, all three output types; split = 0 lets the library choose."""
+    x = wl.activations(35, M + K, M, K, max(1, K // 100), 20.0)
+    g = (wl.weight_codes(35, N + K, N, K), wl.weight_scales(35, N + K, N, mult=0.5))
+    u = (wl.weight_codes(35, N + K + 1, N, K), wl.weight_scales(35, N + K + 1, N, mult=0.5)) if swiglu else None
+    fl = [B.SQAP_L_FORCE_TCGEN05_SPLITK | B.SQAP_L_KSPLIT(split)]
+    check_linear(x, g[0], g[1], up=u, flags_list=fl)
+    check_linear(x, g[0], g[1], up=u, flags_list=fl, bf16=True)
+
+
+def test_linear_cluster_split_k_rejects_more_slices_than_stages():
+    K, N, M = 512, 128, 32         # two stages of 256 codes
+    w = G.pack(wl.weight_codes(36, 1, N, K), wl.weight_scales(36, 1, N))
+    q = torch.zeros(M * K // 2, dtype=torch.uint8, device="cuda")
+    s = torch.ones(M, dtype=torch.float32, device="cuda")
+    out = torch.zeros(M * N, dtype=torch.float16, device="cuda")
+    nb = B.sqap_workspace_bytes(M, N, K)
+    ws = torch.zeros(nb, dtype=torch.uint8, device="cuda")
+    L = B.lib()
+    call = lambda fl: L.sqap_w4a4_linear(q.data_ptr(), s.data_ptr(), M, w.handle, None, out.data_ptr(), N, B.SQAP_FP16, fl,
+                                         ws.data_ptr(), nb, None)
+    assert call(B.SQAP_L_FORCE_TCGEN05_SPLITK | B.SQAP_L_KSPLIT(3)) == B.SQAP_ERR_UNSUPPORTED
+    assert call(B.SQAP_L_FORCE_TCGEN05_SPLITK | B.SQAP_L_KSPLIT(5)) == B.SQAP_ERR_INVALID
+    assert call(B.SQAP_L_KSPLIT(2)) == B.SQAP_ERR_INVALID            # a cluster size without the kernel it belongs to
+    assert call(B.SQAP_L_FORCE_TCGEN05_SPLITK | B.SQAP_L_KSPLIT(2)) == B.SQAP_OK
+    torch.cuda.synchronize()
+    assert B.sqap_device_status() == B.SQAP_OK
+    w.close()
 
 
 @pytest.mark.parametrize("K", [64, 128, 256, 512, 4096])
