@@ -125,10 +125,11 @@ class Layer:
 class Path:
     """Device state of one rank and the step function (all work goes through the C ABI)."""
 
-    def __init__(self, torch, B, device, seed: int):
+    def __init__(self, torch, B, device, seed: int, keep_host_weights: bool = False):
         self.torch, self.B, self.dev = torch, B, device
         t = torch
         inp = wl.config4_inputs(seed=seed, batch=N_OBS)
+        self.inputs_host = inp
         self.x_host = t.from_numpy(inp["x"].reshape(M_FULL, wl.HIDDEN)).pin_memory()
         self.scores_host = t.from_numpy(inp["scores"]).pin_memory()
         self.centers_host = t.from_numpy(inp["centers"]).pin_memory()
@@ -141,9 +142,12 @@ class Path:
             return B.sqap_pack_weights(np.ascontiguousarray(codes), np.ascontiguousarray(scales), N, K)
 
         self.layers = []
+        self.host_weights_b = None      # layer B's codes and scales stay on the host for the untimed oracle check
         for li in range(2):
             wts = wl.config4_weights(seed=seed + 100 * li)
             self.layers.append(Layer(B, pack, wts))
+            if li == 1 and keep_host_weights:
+                self.host_weights_b = wts
             del wts
         M = M_FULL
         f16, u8, f32, i32 = t.float16, t.uint8, t.float32, t.int32
@@ -224,6 +228,61 @@ def time_region(torch, fn, steps: int, world: int):
     return du.max_over_ranks(ms, world, device="cuda")
 
 
+def _within_tolerance(got_bits, ref_bits):
+    """fp16: |got - ref| <= max(1 ulp at ref, 2e-3 |ref|), elementwise."""
+    g = got_bits.view(np.float16).astype(np.float64)
+    r = ref_bits.view(np.float16).astype(np.float64)
+    ulp = np.spacing(np.abs(ref_bits.view(np.float16))).astype(np.float64)
+    return np.isfinite(r) & (np.abs(g - r) <= np.maximum(ulp, 2e-3 * np.abs(r)))
+
+
+def check_step_against_oracle(torch, path: Path, step_fn):
+    """Untimed. Replays the timed step once more and compares what it left on the device with the CPU oracle:
+    the kept-token indices of every observation (bit-exact), the gathered rows (bit-exact), and, for sampled token
+    rows of the pruned layer and of the decode step, every linear of the chain on the input it actually received
+    (the oracle applied to the device's own input of that stage), fp16 within max(1 ulp, 2e-3)."""
+    import oracle
+    oracle.build()
+    t = torch
+    step_fn()
+    t.cuda.synchronize()
+    inp, wts = path.inputs_host, path.host_weights_b
+    bits = lambda a: np.ascontiguousarray(a).view(np.uint16)
+    kept = path.io[0]["kept"].cpu().numpy()
+    kept_o, nk_o = oracle.prune_tokens(path.prune_params, bits(inp["scores"]), inp["centers"])
+    if not (np.array_equal(kept, kept_o) and np.array_equal(path.nkept.cpu().numpy(), nk_o)):
+        return False, "kept indices differ from the oracle"
+    x1_o = oracle.gather_rows(bits(inp["x"]), kept_o, nk_o, ROWS_KEPT).reshape(M_PRUNED, wl.HIDDEN)
+    if not np.array_equal(bits(path.x1.cpu().numpy()), x1_o):
+        return False, "gathered rows differ from the oracle"
+
+    def lin(x_bits, name, rotate=False, up=None):
+        _, s, codes = oracle.quantize_act(np.ascontiguousarray(x_bits), rotate=rotate)
+        acc = oracle.gemm_i32(codes, wts[name + "_codes"])
+        sw = bits(wts[name + "_scales"])
+        if up is None:
+            return oracle.epilogue(acc, s, sw)
+        return oracle.epilogue_swiglu(acc, oracle.gemm_i32(codes, wts[up + "_codes"]), s, sw, bits(wts[up + "_scales"]))
+
+    H = wl.HIDDEN
+    rng = np.random.default_rng(7)
+    # rows 0..15 of the shared qkv / o / h buffers hold the decode step (it ran last), the rest the pruned layer
+    rows_b = np.unique(np.concatenate([[N_OBS, M_PRUNED - 1], rng.integers(N_OBS, M_PRUNED, 4)]))
+    rows_d = np.arange(0, N_OBS, 5)
+    for rows, x_in, d_out, what in ((rows_b, x1_o, path.io[0]["d1"], "pruned layer"),
+                                    (rows_d, bits(path.xdec_host.numpy()), path.io[0]["ddec"], "decode")):
+        idx = t.from_numpy(rows).to(path.dev)
+        get = lambda buf: bits(buf[idx].cpu().numpy())
+        qkv, o, h, d = get(path.qkv), get(path.o), get(path.h), get(d_out)
+        for name, got, ref in (("qkv", qkv, lin(x_in[rows], "qkv", rotate=True)), ("o", o, lin(qkv[:, 2 * H:], "o")),
+                               ("gate/up", h, lin(o, "gate", up="up")), ("down", d, lin(h, "down"))):
+            ok = _within_tolerance(got, ref)
+            if not ok.all():
+                return False, f"{what}, {name}: {int((~ok).sum())} of {ok.size} sampled outputs outside tolerance"
+    return True, (f"kept indices and gathered rows of {N_OBS} observations bit-exact; {len(rows_b)} rows of the pruned layer and "
+                  f"{len(rows_d)} decode rows through all four linears within max(1 ulp, 2e-3) of the oracle")
+
+
 def dominant_gemm_roofline(torch, B, path: Path, steps: int, peaks: dict):
     """The QKV GEMM at M = 4608 (largest single launch), timed alone with CUDA events on its stream.
     The expand pass is skipped (SQAP_L_REUSE_EXPANDED), so the events bracket GEMM launches only."""
@@ -245,13 +304,89 @@ def dominant_gemm_roofline(torch, B, path: Path, steps: int, peaks: dict):
     ops = 2.0 * M * N * K
     achieved = ops / (ms * 1e-3) / 1e12
     peak = 2.0 * peaks["bf16"]       # int8 dense = 2 x bf16 dense (nominal ratio) x the measured bf16 burst figure
-    # traffic: dram__bytes_read.sum + dram__bytes_write.sum of one launch of this kernel at this shape, from the ncu
-    # capture summarised in profiles/w4a4_tc_pair_kernel_qkv_m4608.md (algorithmic bytes: 25.2 MB packed weights
-    # + 18.9 MB int8 activations + 113.2 MB fp16 output = 157.3 MB; part of the output is still in L2 at the end).
+    traffic, traffic_src = profile_traffic("w4a4_tc_pair_kernel_qkv_m4608.md")
     return dict(bound="tensor", kernel="w4a4_tc_pair_kernel: W4A4 linear GEMM, M=4608 N=12288 K=4096 (int8 MMA on CTA "
                                        "pairs, int32 accumulate in tensor memory)",
-                achieved=achieved, peak=peak, unit="TOP/s", frac=achieved / peak, traffic=118.0e6,
-                peak_source=f"2 x bf16 burst ({peaks['source']})", ms_per_launch=ms)
+                achieved=achieved, peak=peak, unit="TOP/s", frac=achieved / peak, traffic=traffic,
+                traffic_source=traffic_src, algorithmic_bytes=N * K // 2 + M * K + 2 * M * N,
+                peak_source=f"2 x bf16 cuBLAS burst ({peaks['source']}); a power-capped library run, not a ceiling",
+                frac_of_nominal_int8=achieved / NOMINAL_INT8_TOPS, nominal_int8_tops=NOMINAL_INT8_TOPS,
+                ms_per_launch=ms)
+
+
+NOMINAL_INT8_TOPS = 4500.0      # B200 dense int8, nominal
+INT8_MAC_PER_CLK_SM = 8192      # what one SM's tensor pipe retires (measured: 128 cycles per 128x256x32 MMA)
+
+
+def pipe_peak_tops(sm_mhz, sms=148):
+    """int8 tensor-pipe ceiling at a given SM clock: 8192 MAC per clock and SM."""
+    return 2.0 * INT8_MAC_PER_CLK_SM * sms * sm_mhz * 1e6 / 1e12
+
+
+def profile_traffic(name):
+    """dram__bytes_read.sum + dram__bytes_write.sum of launch 0 from an ncu summary under profiles/ (bytes), or
+    (None, reason) when the file or the counters are missing."""
+    import re
+    path = os.path.join(ROOT, "profiles", name)
+    try:
+        text = open(path).read()
+    except OSError:
+        return None, "no ncu summary for this kernel"
+    unit = {"byte": 1.0, "Kbyte": 1e3, "Mbyte": 1e6, "Gbyte": 1e9}
+    tot = 0.0
+    for key in ("dram__bytes_read.sum", "dram__bytes_write.sum"):
+        m = re.search(r"`" + re.escape(key) + r"`\)\s*\|\s*([0-9.]+)\s*([KMG]?byte)", text)
+        if not m:
+            return None, "counters not found in profiles/" + name
+        tot += float(m.group(1)) * unit[m.group(2)]
+    return tot, "profiles/" + name + " (launch 0)"
+
+
+def hbm_kernel_rooflines(torch, B, path: Path, peaks: dict):
+    """The HBM-bound kernels of the step, each timed alone (CUDA-graph replays over buffers rotating through more
+    than the L2 capacity): algorithmic bytes / time / measured HBM copy bandwidth."""
+    t, dev = torch, path.dev
+    H = wl.HIDDEN
+    hbm = peaks["hbm_gbs"]
+    out = []
+    gen = t.Generator(device=dev)
+    gen.manual_seed(99)
+
+    def add(kernel, nbytes, us):
+        ach = nbytes / (us * 1e-6) / 1e9
+        out.append(dict(kernel=kernel, bound="hbm", bytes=nbytes, us=us, achieved=ach, peak=hbm, unit="GB/s", frac=ach / hbm))
+
+    n = 5                                               # 5 x 37.7 MB of activations > L2
+    xs = [t.randn(M_FULL, H, device=dev, generator=gen).to(t.float16) for _ in range(n)]
+    for rot in (False, True):
+        fl = B.SQAP_Q_ROTATE if rot else 0
+        us = graph_time_us(t, lambda i: B.sqap_quantize_act(xs[i % n], M_FULL, H, H, None, fl, path.q, path.sx), reps=10)
+        add("quantize_act" + (" + Hadamard" if rot else "") + f", M={M_FULL} K={H}", M_FULL * H * 2.5 + 4 * M_FULL, us)
+    p = path.prune_params
+    io = path.io[0]
+    us_sel = graph_time_us(t, lambda i: B.sqap_prune_tokens(p, io["scores"], io["centers"], None, 0, 0, None, 0, 0,
+                                                            io["kept"], path.nkept), reps=8)
+    us_all = graph_time_us(t, lambda i: B.sqap_prune_tokens(p, io["scores"], io["centers"], xs[i % n], H, H, path.x1, H,
+                                                            ROWS_KEPT, io["kept"], path.nkept), reps=10)
+    add(f"gather_rows, {N_OBS} x {ROWS_KEPT} rows x {H} (prune call minus its selection kernel)", 2 * M_PRUNED * H * 2,
+        max(us_all - us_sel, 1e-3))
+    out.append(dict(kernel="prune_select (top-k U ring U FPS, compaction)", bound="latency", us=us_sel,
+                    note="serial farthest-point steps; no bandwidth fraction applies"))
+    del xs
+    # the M = 16 weight streamer on the QKV shape, over more weight matrices than the L2 holds
+    codes = t.randint(-8, 8, (wl.QKV, H), dtype=t.int8, device=dev, generator=gen)
+    scales = (t.rand(wl.QKV, device=dev, generator=gen) * 0.015 + 0.005).to(t.float16)
+    ws = [B.sqap_pack_weights(codes, scales, wl.QKV, H) for _ in range(7)]
+    t.cuda.synchronize()
+    del codes
+    sc_ptr = path.ws.data_ptr() + B.sqap_workspace_bytes(N_OBS, wl.QKV, H)
+    B.sqap_quantize_linear(path.xdec, N_OBS, H, None, 0, ws[0], None, path.qkv, wl.QKV, B.SQAP_FP16, 0, path.ws, path.ws_bytes)
+    us = graph_time_us(t, lambda i: B.sqap_w4a4_linear(path.ws, sc_ptr, N_OBS, ws[i % 7], None, path.qkv, wl.QKV, B.SQAP_FP16,
+                                                       B.SQAP_L_REUSE_EXPANDED, path.ws, path.ws_bytes), reps=14)
+    add(f"w4a4_mma_kernel (weight streamer), M={N_OBS} N={wl.QKV} K={H}", wl.QKV * H // 2 + N_OBS * H + 2 * N_OBS * wl.QKV, us)
+    for w in ws:
+        w.close()
+    return out
 
 
 def cpu_baseline(seconds_budget: float = 15.0):
@@ -306,7 +441,8 @@ def run_ours(args):
     device = torch.device("cuda", local_rank)
     B.lib()
     peaks = measured_peaks()
-    path = Path(torch, B, device, seed=4 + 1000 * rank)
+    sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
+    path = Path(torch, B, device, seed=4 + 1000 * rank, keep_host_weights=(rank == 0 and not args.no_parity_check))
     path.upload()
     torch.cuda.synchronize()
 
@@ -380,9 +516,27 @@ def run_ours(args):
         e2e_step()
     torch.cuda.synchronize()
     ms_e2e = time_region(torch, e2e_region, 1, world)
+    # A second, long timed region of the same replayed step: what the step does over seconds, under the power cap
+    # (the regime the sustained library figure describes). It does not change `value`.
+    sus_steps = int(min(max(np.ceil(args.sustain_s * 1e3 / (ms / args.steps)), 1), 20000)) if args.sustain_s > 0 else 0
+    sus = None
+    if sus_steps:
+        sampler2 = ClockSampler(local_rank)
+        if rank == 0:
+            sampler2.start()
+        ms_sus = time_region(torch, step_fn, sus_steps, world)
+        clocks_sus = sampler2.stop() if rank == 0 else None
+        sus = (ms_sus, sus_steps, clocks_sus)
     roof = dominant_gemm_roofline(torch, B, path, max(args.steps, 10), peaks) if rank == 0 else None
+    roof_hbm = hbm_kernel_rooflines(torch, B, path, peaks) if rank == 0 else None
     if B.sqap_device_status() != B.SQAP_OK:
         raise SystemExit("bench.py: a kernel reported an expired bounded wait")
+    parity = None
+    if rank == 0 and not args.no_parity_check:
+        ok, what = check_step_against_oracle(torch, path, step_fn)
+        if not ok:
+            raise SystemExit("bench.py: the timed step does not match the CPU oracle: " + what)
+        parity = what
 
     ms_step = ms / args.steps
     tops = world * STEP_OPS / (ms_step * 1e-3) / 1e12
@@ -405,8 +559,29 @@ def run_ours(args):
             "gpu_launches": int(launches), "launch_mode": "eager" if args.no_graph else "cuda_graph replay",
             "clocks": clocks,
             "roofline": roof,
+            "roofline_hbm": roof_hbm,
             "cpu_baseline": cpu,
+            "parity_checked": parity is not None, "parity": parity,
         }
+        mhz = clocks.get("sm_mhz") if clocks else None
+        if mhz:
+            # the tensor pipe itself, at the clock the timed region ran at (8192 int8 MAC per clock and SM)
+            line["ms_x_mhz"] = ms_step * mhz
+            line["roofline"]["pipe_peak_at_sampled_clock"] = pipe_peak_tops(mhz, sm_count)
+            line["roofline"]["frac_of_pipe"] = roof["achieved"] / pipe_peak_tops(mhz, sm_count)
+            line["value_frac_of_pipe"] = tops / world / pipe_peak_tops(mhz, sm_count)
+        if sus:
+            ms_sus, sus_steps, clocks_sus = sus
+            ms_s = ms_sus / sus_steps
+            tops_s = world * STEP_OPS / (ms_s * 1e-3) / 1e12
+            line["sustained"] = {"seconds": ms_sus * 1e-3, "steps": sus_steps, "ms_per_step": ms_s, "value": tops_s,
+                                 "unit": "TOPS", "clocks": clocks_sus,
+                                 "frac_sustained": tops_s / world / (2.0 * peaks["bf16_sustained"]),
+                                 "peak_sustained": 2.0 * peaks["bf16_sustained"],
+                                 "peak_source": f"2 x bf16 cuBLAS sustained ({peaks['source']})"}
+            if clocks_sus and clocks_sus.get("sm_mhz"):
+                line["sustained"]["ms_x_mhz"] = ms_s * clocks_sus["sm_mhz"]
+                line["sustained"]["frac_of_pipe"] = tops_s / world / pipe_peak_tops(clocks_sus["sm_mhz"], sm_count)
         print(json.dumps(line))
     du.finish(world)
 
@@ -624,7 +799,8 @@ def run_stack(args):
         t.cuda.synchronize()
         return w
 
-    n_layers = 32
+    from paper_2509_09090_b200.stack import Stack
+    n_layers = wl.N_LAYERS
     layers = [dict(qkv=rand_w(Q, H), o=rand_w(H, H), gate=rand_w(F, H), up=rand_w(F, H), down=rand_w(H, F))
               for _ in range(n_layers)]
     inp = wl.config4_inputs(seed=3, batch=1)
@@ -633,38 +809,10 @@ def run_stack(args):
     xdec = t.from_numpy(wl.activations(3, wl.T_X2, 7, H, 41, 30.0)).to(dev)
     keep = 128
     rows_kept = 32 + keep
-    x1 = t.empty(rows_kept, H, dtype=t.float16, device=dev)
-    kept = t.empty(1, wl.ROWS, dtype=t.int32, device=dev)
-    nk = t.empty(1, dtype=t.int32, device=dev)
-    p = wl.prune_params(1, wl.ROWS, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32, keep // 2, keep, ring_radius=1)
     M = wl.ROWS
-    qkv = t.empty(M, Q, dtype=t.float16, device=dev)
-    o = t.empty(M, H, dtype=t.float16, device=dev)
-    h = t.empty(M, F, dtype=t.float16, device=dev)
-    d = t.empty(n_layers, M, H, dtype=t.float16, device=dev)
-    nb = B.sqap_quantize_linear_workspace_bytes(M, Q, F)
-    ws = t.empty(nb, dtype=t.uint8, device=dev)
-
-    def lin(xp, m, ldx, w, w_up, out, rot=False):
-        B.sqap_quantize_linear(xp, m, ldx, None, B.SQAP_Q_ROTATE if rot else 0, w, w_up, out, out.shape[-1], B.SQAP_FP16,
-                               0, ws, nb)
-
-    def layer(xin, m, L, dout):
-        lin(xin.data_ptr(), m, H, L["qkv"], None, qkv, rot=True)
-        lin(qkv.data_ptr() + 2 * 2 * H, m, Q, L["o"], None, o)
-        lin(o.data_ptr(), m, H, L["gate"], L["up"], h)
-        lin(h.data_ptr(), m, F, L["down"], None, dout)
-
-    def prefill():
-        for li in range(n_layers):
-            if li == 2:
-                B.sqap_prune_tokens(p, sc, ce, x, H, H, x1, H, rows_kept, kept, nk)
-            layer(x if li < 2 else x1, M if li < 2 else rows_kept, layers[li], d[li])
-
-    def decode():
-        for step in range(7):
-            for li in range(n_layers):
-                layer(xdec[step:step + 1], 1, layers[li], d[li])
+    st = Stack(t, B, dev, layers, keep=keep, k_attn=keep // 2, ring_radius=1, n_decode=7)
+    prefill = lambda: st.prefill(x, sc, ce)
+    decode = lambda: st.decode(xdec)
 
     def timed(fn, reps):
         fn()
@@ -745,6 +893,44 @@ def run_single_kernel(args):
     print(json.dumps({"profiling_run": args.kernel, "launches": B.sqap_kernel_launch_count()}))
 
 
+def spawn_ranks(n: int) -> int:
+    """`python bench.py --gpus N` without a launcher: start the N ranks (one process per GPU, rendezvous on
+    127.0.0.1), pass rank 0's output through and return the worst exit code."""
+    import socket
+    with socket.socket() as sk:
+        sk.bind(("127.0.0.1", 0))
+        port = sk.getsockname()[1]
+    procs = []
+    for r in range(n):
+        env = dict(os.environ, RANK=str(r), LOCAL_RANK=str(r), WORLD_SIZE=str(n), MASTER_ADDR="127.0.0.1",
+                   MASTER_PORT=str(port))
+        procs.append(subprocess.Popen([sys.executable, os.path.abspath(__file__)] + sys.argv[1:], env=env,
+                                      stdout=None if r == 0 else subprocess.DEVNULL))
+    rc = 0
+    for pr in procs:
+        rc = max(rc, abs(pr.wait()))
+    return rc
+
+
+def run_stub(args):
+    """The multi-rank plumbing of run_ours around a CPU stand-in for the step (no GPU, no kernels): process-group
+    start-up from the environment, barrier-bracketed timing, maximum over ranks, one JSON line from rank 0."""
+    rank, _, world = du.init(args.stub_backend)
+    first, cnt = du.shard_observations(N_OBS * world, world, rank)
+    du.barrier(world)
+    t0 = time.perf_counter()
+    acc = 0
+    for _ in range(args.steps):
+        acc += sum(range(1000 * (rank + 1)))
+    ms = du.max_over_ranks((time.perf_counter() - t0) * 1e3, world)
+    total = du.sum_over_ranks(cnt, world)
+    du.barrier(world)
+    if rank == 0:
+        print(json.dumps({"stub": True, "n_gpus": world, "steps": args.steps, "ms_per_step": ms / max(args.steps, 1),
+                          "observations": int(total), "scaling": "weak"}))
+    du.finish(world)
+
+
 def main():
     ap = argparse.ArgumentParser()
     ap.add_argument("--gpus", type=int, default=1)
@@ -752,6 +938,11 @@ def main():
     ap.add_argument("--warmup", type=int, default=3)
     ap.add_argument("--impl", default="ours", choices=["ours", "reference"])
     ap.add_argument("--no-cpu-baseline", action="store_true")
+    ap.add_argument("--no-parity-check", action="store_true", help="skip the untimed oracle check of the replayed step")
+    ap.add_argument("--sustain-s", type=float, default=2.0,
+                    help="length in seconds of the second, sustained timed region (0: none)")
+    ap.add_argument("--stub-backend", default=None, choices=["gloo"],
+                    help="plumbing test: run the rank start-up, barriers and max-over-ranks timing around a CPU stub step")
     ap.add_argument("--no-graph", action="store_true", help="issue the step's launches eagerly instead of replaying a CUDA graph")
     ap.add_argument("--detail", action="store_true",
                     help="time every kernel of the path alone at the workload's shapes (one JSON table, no bench line)")
@@ -760,7 +951,11 @@ def main():
     ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "stream", "midm", "quantize", "prune"],
                     help="profiling aid: launch only this kernel --steps times (no bench line)")
     args = ap.parse_args()
-    if args.stack:
+    if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
+        raise SystemExit(spawn_ranks(args.gpus))
+    if args.stub_backend:
+        run_stub(args)
+    elif args.stack:
         run_stack(args)
     elif args.detail:
         run_detail(args)

@@ -86,7 +86,7 @@ inline bool aligned16(const void* p) { return (reinterpret_cast<uintptr_t>(p) & 
 // scales only, which are immutable after packing). Since these kernels release their dependents before their own
 // wait, up to three kernels of a chain can be resident at once; the rule is what keeps the workspace (expanded
 // codes, row sums, scales), which consecutive calls rewrite, and the activations free of races.
-constexpr int PDL_MAX_ROWS = 32;   // the quantizers launch this way up to here (the row counts of decode steps)
+constexpr int PDL_MAX_ROWS = 32;   // the row counts of decode steps (the Hadamard quantizer treats them specially)
 #ifdef __CUDACC__
 __device__ __forceinline__ void pdl_wait() { asm volatile("griddepcontrol.wait;" ::: "memory"); }
 __device__ __forceinline__ void pdl_launch_dependents() { asm volatile("griddepcontrol.launch_dependents;" ::: "memory"); }

@@ -37,21 +37,23 @@ constexpr int S_MAX = 8;                  // TMA ring (packed weights + activati
 constexpr int U_MAX = 4;                  // ring of unpacked weight tiles in tensor memory: 2 to 4
 constexpr int KSPLIT_MAX = 4;             // CTAs per cluster
 constexpr int W_BYTES = BM * BK / 2;      // 16 KB: a stage's packed weights, 128 rows of 128 bytes
-constexpr int RING_BYTES = 206 * 1024;    // stage s: [weights][tokens half 0][tokens half 1]; later the exchange buffer
+constexpr int RING_BYTES = 222 * 1024;    // stage s: [weights][tokens half 0][tokens half 1]; after the main loop:
+constexpr int OFF_XCHG = 0;               //   the exchange buffer (partial accumulators, at most 120 KB)
+constexpr int OFF_STAGE = 128 * 1024;     //   and the staging of the coalesced epilogue: 3 groups x 2 buffers x 4 KB
 constexpr int OFF_BAR = RING_BYTES;
 constexpr int OFF_TOK = OFF_BAR + 512;    // per-token epilogue constants, BN_MAX x 8 bytes
-constexpr int OFF_STAGE = OFF_TOK + BN_MAX * 8;       // staging of the coalesced epilogue (tc_common.cuh)
-constexpr int SMEM_BYTES = OFF_STAGE + EPI_STAGE_TOTAL + 1024;  // + slack for 1024-byte alignment
+constexpr int SMEM_BYTES = OFF_TOK + BN_MAX * 8 + 1024;  // + slack for 1024-byte alignment
 constexpr int A_COLS = BK / 4;            // 64 columns hold 256 int8 per lane
 constexpr int TMEM_A_COL = 256;           // accumulator: columns [0, BN); weight tiles from here
-constexpr int EPI_WARPS = 8;
-constexpr int THREADS = 32 * (6 + EPI_WARPS);
+constexpr int THREADS = 32 * 14;          // as the other tcgen05 kernels (warps 6-13 have no main-loop role here)
+constexpr int EPI_GROUPS = 3;             // groups of four warps (one per tensor-memory lane quadrant) in the epilogue
 constexpr int CHUNK_BYTES = BM * 16 * 4;  // one 16-token chunk of a partial accumulator: 128 rows x 16 int32
 static_assert(TMEM_A_COL + U_MAX * A_COLS <= 512 && BN_MAX <= TMEM_A_COL, "tensor memory budget");
 static_assert(SMEM_BYTES <= 227 * 1024, "shared memory budget");
 static_assert(8 * (3 * S_MAX + U_MAX + 1) + 16 <= 512, "barrier block");
 // every CTA receives ksplit partials of at most ceil(chunks / ksplit) chunks
-static_assert((BN_MAX / 16 + KSPLIT_MAX - 1) * CHUNK_BYTES <= RING_BYTES, "exchange buffer fits the ring");
+static_assert((BN_MAX / 16 + KSPLIT_MAX - 1) * CHUNK_BYTES <= OFF_STAGE, "exchange buffer ends before the staging");
+static_assert(OFF_STAGE + EPI_GROUPS * 2 * EPI_STAGE_BYTES <= RING_BYTES, "staging fits the ring");
 
 inline __host__ __device__ int stage_bytes_for(int BN) { return W_BYTES + 2 * BN * BKH; }
 
@@ -127,18 +129,44 @@ w4a4_tc_splitk_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
     const int ks_begin = rank * k_steps / ksplit, ks_end = (rank + 1) * k_steps / ksplit;   // ksplit <= k_steps: never empty
     const int my_steps = ks_end - ks_begin;
 
-    if (threadIdx.x == 0) {
-        for (int s = 0; s < S; ++s) {
-            mbar_init(full(s), 1);
-            mbar_init(done(s), 1);
-            mbar_init(wp_empty(s), 4);
+    // Set-up. Warp 0 initialises the barriers and at once issues the WEIGHT loads of its first stages (fresh ring slots
+    // need no waiting), so that the first weights are on their way while tensor memory is allocated and the CTA
+    // meets, and, when this kernel was launched as a programmatic dependent, while the kernel before it in the
+    // stream is still running: packed weights never change, whereas the tokens are that kernel's output and are
+    // fetched after the dependency wait.
+    auto issue_weights = [&](int ks, int s, uint32_t issue) {
+        mbar_expect_tx_if(full(s), stage_bytes, issue);   // the whole stage's bytes: the tokens follow
+        const uint32_t wp = w_addr(s);
+        if (a.swiglu) {
+            tma_load_2d_if(wp, &tm_w, ks * (BK / 2), n0 / 2, full(s), issue);
+            tma_load_2d_if(wp + W_BYTES / 2, &tm_w_up, ks * (BK / 2), n0 / 2, full(s), issue);
+        } else {
+            tma_load_2d_if(wp, &tm_w, ks * (BK / 2), n0, full(s), issue);
         }
-        for (int j = 0; j < U; ++j) mbar_init(a_full(j), 4);
-        mbar_init(acc_full, 1);
-        abort_flag[0] = 0;
-        abort_flag[1] = 0;  // always-zero word for waits that must ignore the abort request
-        asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+    };
+    auto issue_tokens = [&](int ks, int s, uint32_t issue) {
+#pragma unroll
+        for (int h = 0; h < 2; ++h) tma_load_2d_if(x_addr(s, h), &tm_x, ks * BK + h * BKH, m0, full(s), issue);
+    };
+    const int pre = my_steps < S ? my_steps : S;   // stages issued before the set-up barrier
+    if (warp == 0) {
+        if (lane == 0) {
+            for (int s = 0; s < S; ++s) {
+                mbar_init(full(s), 1);
+                mbar_init(done(s), 1);
+                mbar_init(wp_empty(s), 4);
+            }
+            for (int j = 0; j < U; ++j) mbar_init(a_full(j), 4);
+            mbar_init(acc_full, 1);
+            abort_flag[0] = 0;
+            abort_flag[1] = 0;  // always-zero word for waits that must ignore the abort request
+            asm volatile("fence.mbarrier_init.release.cluster;" ::: "memory");
+        }
+        __syncwarp();
+        const uint32_t issue = elect_one();
+        for (int it = 0; it < pre; ++it) issue_weights(ks_begin + it, it, issue);
     }
+    pdl_launch_dependents();
     if (warp == 1) {
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
@@ -148,26 +176,20 @@ w4a4_tc_splitk_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
+    pdl_wait();   // the activations, their sums and scales are read, and the output written, only from here on
 
     if (warp == 0) {
         // ---------------- TMA producer: the whole warp walks the loop, one elected lane issues
         const uint32_t issue = elect_one();
-        int s = 0;
-        uint32_t ph = 0;
-        int it = 0;
-        for (int ks = ks_begin; ks < ks_end; ++ks, ++it) {
+        for (int it = 0; it < pre; ++it) issue_tokens(ks_begin + it, it, issue);
+        int s = pre == S ? 0 : pre;
+        uint32_t ph = pre == S ? 1u : 0u;
+        int it = pre;
+        for (; it < my_steps; ++it) {
             const bool ok = mbar_wait(done(s), ph ^ 1u, abort_flag) && mbar_wait(wp_empty(s), ph ^ 1u, abort_flag);
             if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-            mbar_expect_tx_if(full(s), stage_bytes, issue);
-            const uint32_t wp = w_addr(s);
-            if (a.swiglu) {
-                tma_load_2d_if(wp, &tm_w, ks * (BK / 2), n0 / 2, full(s), issue);
-                tma_load_2d_if(wp + W_BYTES / 2, &tm_w_up, ks * (BK / 2), n0 / 2, full(s), issue);
-            } else {
-                tma_load_2d_if(wp, &tm_w, ks * (BK / 2), n0, full(s), issue);
-            }
-#pragma unroll
-            for (int h = 0; h < 2; ++h) tma_load_2d_if(x_addr(s, h), &tm_x, ks * BK + h * BKH, m0, full(s), issue);
+            issue_weights(ks_begin + it, s, issue);
+            issue_tokens(ks_begin + it, s, issue);
             if (++s == S) { s = 0; ph ^= 1u; }
         }
         if (failed && issue) {
@@ -249,53 +271,51 @@ w4a4_tc_splitk_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
         }
     }
 
-    // ---------------- reduce-scatter of the partial accumulators, then the epilogue
+    // ---------------- reduce-scatter of the partial accumulators, then the epilogue: every warp takes part
     // Chunk c (tokens 16c .. 16c+15 of the tile) belongs to CTA c % ksplit, which keeps the partials of its chunk
     // number c / ksplit from source CTA r at  (r * own_max + c / ksplit) * CHUNK_BYTES, as four planes of
     // [128 rows][16 bytes] (plane q = tokens 4q .. 4q+3): thread = row, so a warp's accesses are contiguous.
+    // The work of this part is a chain of short latencies per 16-token chunk (tensor-memory load, distributed
+    // store; later shared-memory loads, a few conversions and multiplies, a staging store, a barrier, the global
+    // store): measured at several hundred cycles per chunk and warp whatever the instruction mix, so it is spread
+    // over as many warps as tensor memory's lane quadrants allow: three groups of four warps (warp % 4 = quadrant).
     const int chunks = a.BN >> 4;
     const int own_max = (chunks + ksplit - 1) / ksplit;
-    const int quad = warp & 3, half = (warp - 6) >> 2;   // epilogue warps: tensor-memory quadrant; which half of the chunks
+    const int quad = warp & 3, group = warp >> 2;   // warps 12, 13 (group 3) only keep the barriers company
     const int row = quad * 32 + lane;
-    if (warp >= 6) {
-        // the tile's per-token constants
-        int2* tok = reinterpret_cast<int2*>(sm + OFF_TOK);
-        const int et = static_cast<int>(threadIdx.x) - 6 * 32;
-        if (et < a.BN) {
-            const int m = m0 + et;
-            tok[et] = m < a.M ? make_int2(__ldg(a.bias_sum + m) << 7, __float_as_int(__ldg(a.act_scales + m))) : make_int2(0, 0);
-        }
-        // all epilogue warps agree on failure, so that none of them reads an accumulator that is not complete
-        if (bar_or(1, 32 * EPI_WARPS, !mbar_wait(acc_full, 0u, abort_flag))) failed = true;
-        tc_fence_after();
+    int2* tok = reinterpret_cast<int2*>(sm + OFF_TOK);
+    if (static_cast<int>(threadIdx.x) < a.BN) {   // the tile's per-token constants
+        const int m = m0 + static_cast<int>(threadIdx.x);
+        tok[threadIdx.x] = m < a.M ? make_int2(__ldg(a.bias_sum + m) << 7, __float_as_int(__ldg(a.act_scales + m))) : make_int2(0, 0);
     }
+    if (!failed && !mbar_wait(acc_full, 0u, abort_flag)) failed = true;
     if (failed) {
         *abort_flag = 1;
         atomicOr(a.status, SQAP_ERR_TIMEOUT);
     }
-    __syncwarp();
+    failed = __syncthreads_or(failed ? 1 : 0) != 0;   // from here on the whole CTA agrees; tok is complete
+    tc_fence_after();
     cluster_sync_all();   // #1: every CTA's MMAs are done (or given up): the rings are idle and may receive partials
-    if (warp >= 6 && !failed) {
+    if (group < EPI_GROUPS && !failed) {
         const uint32_t taddr = tmem_base + (static_cast<uint32_t>(quad * 32) << 16);
-        for (int c = half; c < chunks; c += 2) {
+        for (int c = group; c < chunks; c += EPI_GROUPS) {
             uint32_t v[16];
             tc_ld16(taddr + 16 * c, v);
-            const uint32_t dst = map_to_cta(base + static_cast<uint32_t>((rank * own_max + c / ksplit) * CHUNK_BYTES + row * 16),
+            const uint32_t dst = map_to_cta(base + static_cast<uint32_t>(OFF_XCHG + (rank * own_max + c / ksplit) * CHUNK_BYTES + row * 16),
                                             static_cast<uint32_t>(c % ksplit));
             tc_wait_ld();
 #pragma unroll
             for (int q = 0; q < 4; ++q) st_cluster_v4(dst + q * (BM * 16), v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3]);
         }
-        tc_fence_before();
     }
+    tc_fence_before();
     __syncwarp();
     cluster_sync_all();   // #2: all partials have arrived; nobody touches another CTA's shared memory from here on
     if (warp == 1) {
         tc_fence_after();
         asm volatile("tcgen05.dealloc.cta_group::1.sync.aligned.b32 %0, 512;" ::"r"(tmem_base) : "memory");
     }
-    if (warp >= 6 && !failed) {
-        const int2* tok = reinterpret_cast<const int2*>(sm + OFF_TOK);
+    if (group < EPI_GROUPS && !failed) {
         int n;
         float sw;
         bool n_ok;
@@ -309,33 +329,34 @@ w4a4_tc_splitk_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_con
             sw = n_ok ? __half2float(a.w_scales[n]) : 0.0f;
         }
         const int own = (chunks - rank + ksplit - 1) / ksplit;   // chunks rank, rank + ksplit, ...
-        for (int lc = half; lc < own; lc += 2) {
+        const bool odd = (lane & 16) != 0;
+        const int ch = a.swiglu ? quad * 16 + (lane & 15) : row, n_tile0 = a.swiglu ? n0 / 2 : n0;
+        for (int lc = group, turn = 0; lc < own; lc += EPI_GROUPS, turn ^= 1) {
             const int c = lc * ksplit + rank;
+            const int m_first = m0 + 16 * c;
+            const int4* t4 = reinterpret_cast<const int4*>(tok + 16 * c);
+            const uint8_t* part = sm + OFF_XCHG + lc * CHUNK_BYTES + row * 16;
             uint32_t v[16];
 #pragma unroll
             for (int i = 0; i < 16; ++i) v[i] = 0;
             for (int r = 0; r < ksplit; ++r) {
-                const uint8_t* src = sm + (r * own_max + lc) * CHUNK_BYTES + row * 16;
 #pragma unroll
                 for (int q = 0; q < 4; ++q) {
-                    const uint4 p = *reinterpret_cast<const uint4*>(src + q * (BM * 16));
+                    const uint4 p = *reinterpret_cast<const uint4*>(part + r * own_max * CHUNK_BYTES + q * (BM * 16));
                     v[4 * q] += p.x; v[4 * q + 1] += p.y; v[4 * q + 2] += p.z; v[4 * q + 3] += p.w;
                 }
             }
-            const int4* t4 = reinterpret_cast<const int4*>(tok + 16 * c);
-            const int m_first = m0 + 16 * c;
             // fp16 / bf16: through shared memory, 16 bytes per thread to global memory; raw int32 (checking): directly
-            const int tid_half = static_cast<int>(threadIdx.x) - (6 + 4 * half) * 32;
-            uint8_t* stage = sm + OFF_STAGE + (half * 2 + ((lc >> 1) & 1)) * EPI_STAGE_BYTES;
+            uint8_t* stage = sm + OFF_STAGE + (group * 2 + turn) * EPI_STAGE_BYTES;
             if (a.swiglu) {
-                const int ch = quad * 16 + (lane & 15);
-                if (a.out_dtype == SQAP_FP16) epilogue_chunk_coalesced<SQAP_FP16, true>(a, v, m_first, n0 / 2, ch, sw, lane, t4, stage, tid_half, 2 + half);
-                else epilogue_chunk_coalesced<SQAP_BF16, true>(a, v, m_first, n0 / 2, ch, sw, lane, t4, stage, tid_half, 2 + half);
+                if (a.out_dtype == SQAP_FP16) epilogue_chunk_coalesced<SQAP_FP16, true>(a, v, m_first, n_tile0, ch, sw, lane, t4, stage, row, 2 + group);
+                else epilogue_chunk_coalesced<SQAP_BF16, true>(a, v, m_first, n_tile0, ch, sw, lane, t4, stage, row, 2 + group);
             } else {
-                if (a.out_dtype == SQAP_FP16) epilogue_chunk_coalesced<SQAP_FP16, false>(a, v, m_first, n0, row, sw, lane, t4, stage, tid_half, 2 + half);
-                else if (a.out_dtype == SQAP_BF16) epilogue_chunk_coalesced<SQAP_BF16, false>(a, v, m_first, n0, row, sw, lane, t4, stage, tid_half, 2 + half);
+                if (a.out_dtype == SQAP_FP16) epilogue_chunk_coalesced<SQAP_FP16, false>(a, v, m_first, n_tile0, ch, sw, lane, t4, stage, row, 2 + group);
+                else if (a.out_dtype == SQAP_BF16) epilogue_chunk_coalesced<SQAP_BF16, false>(a, v, m_first, n_tile0, ch, sw, lane, t4, stage, row, 2 + group);
                 else epilogue_chunk<SQAP_I32, false, 1>(a, v, m_first, n, n_ok, sw, lane, t4);
             }
+            (void)odd;
         }
     }
 }
@@ -446,13 +467,15 @@ sqap_status launch_linear_tcgen05_splitk(const LinearArgs& a, int forced_split, 
     cfg.blockDim = dim3(THREADS);
     cfg.dynamicSmemBytes = SMEM_BYTES;
     cfg.stream = s;
-    cudaLaunchAttribute attr;
-    attr.id = cudaLaunchAttributeClusterDimension;
-    attr.val.clusterDim.x = static_cast<unsigned>(ksplit);
-    attr.val.clusterDim.y = 1;
-    attr.val.clusterDim.z = 1;
-    cfg.attrs = &attr;
-    cfg.numAttrs = 1;
+    cudaLaunchAttribute attr[2];
+    attr[0].id = cudaLaunchAttributeClusterDimension;
+    attr[0].val.clusterDim.x = static_cast<unsigned>(ksplit);
+    attr[0].val.clusterDim.y = 1;
+    attr[0].val.clusterDim.z = 1;
+    attr[1].id = cudaLaunchAttributeProgrammaticStreamSerialization;   // see launch_dependent() in common.cuh
+    attr[1].val.programmaticStreamSerializationAllowed = 1;
+    cfg.attrs = attr;
+    cfg.numAttrs = 2;
     const cudaError_t e = cudaLaunchKernelEx(&cfg, w4a4_tc_splitk_kernel, tm_w, tm_u, tm_x, k, ksplit);
     if (e != cudaSuccess) {
         note_cuda_error(e);

@@ -131,11 +131,15 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
         asm volatile("tcgen05.alloc.cta_group::1.sync.aligned.shared::cta.b32 [%0], 512;" ::"r"(smem_u32(const_cast<uint32_t*>(tmem_slot))) : "memory");
         asm volatile("tcgen05.relinquish_alloc_permit.cta_group::1.sync.aligned;" ::: "memory");
     }
+    pdl_launch_dependents();   // the next kernel of the stream may start its own set-up (it waits before it touches data)
     tc_fence_before();
     __syncthreads();
     tc_fence_after();
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
+    // Everything above is independent of the kernel before this one in the stream; its output (the activations,
+    // their sums and scales) is read, and this kernel's output written, only from here on.
+    pdl_wait();
 
     if (warp == 0) {
         // ---------------- TMA producer: the whole warp walks the loop, one elected lane issues
@@ -382,7 +386,8 @@ sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s) {
     if (st != SQAP_OK) return st;
     const int tiles = k.m_tiles * k.n_tiles;
     const int grid = tiles < sm_count() ? tiles : sm_count();
-    w4a4_tc_ts_kernel<<<grid, THREADS, SMEM_BYTES, s>>>(tm_w, tm_u, tm_x, k);
+    const cudaError_t e = launch_dependent(w4a4_tc_ts_kernel, dim3(grid), dim3(THREADS), SMEM_BYTES, s, tm_w, tm_u, tm_x, k);
+    if (e != cudaSuccess) note_cuda_error(e);
     count_launch();
     return check_launch();
 }

@@ -177,13 +177,9 @@ template <int SINK, int G>
 static void launch_plain(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, const QuantOut& o,
                          cudaStream_t s) {
     constexpr int ROWS = QUANT_THREADS / G;
-    if (M <= PDL_MAX_ROWS) {
-        const cudaError_t e = launch_dependent(quantize_rows_kernel<SINK, G>, dim3((M + ROWS - 1) / ROWS), dim3(QUANT_THREADS), 0, s,
-                                               x, M, K, ldx, row_index, o);
-        if (e != cudaSuccess) note_cuda_error(e);
-        return;
-    }
-    quantize_rows_kernel<SINK, G><<<(M + ROWS - 1) / ROWS, QUANT_THREADS, 0, s>>>(x, M, K, ldx, row_index, o);
+    const cudaError_t e = launch_dependent(quantize_rows_kernel<SINK, G>, dim3((M + ROWS - 1) / ROWS), dim3(QUANT_THREADS), 0, s,
+                                           x, M, K, ldx, row_index, o);
+    if (e != cudaSuccess) note_cuda_error(e);
 }
 
 // ---------------------------------------------------------------------------------------------
@@ -361,9 +357,11 @@ __global__ void __launch_bounds__(R4K_THREADS, 2) quantize_rotate4096_kernel(con
     extern __shared__ __align__(16) uint8_t smem_raw[];
     __shared__ float red_f[R4K_ROWS][2];
     __shared__ int red_i[R4K_ROWS][2];
-    // With more than one CTA, letting the next kernel in early costs more than it saves: this kernel's CTAs are
-    // large, so the SMs they sit on take the streamer's CTAs late, and those then finish last (measured at 16 rows).
-    if (M <= R4K_ROWS) pdl_launch_dependents();
+    // With a handful of CTAs, letting the next kernel in early costs more than it saves: this kernel's CTAs are
+    // large, so the SMs they sit on take the weight streamer's CTAs late, and those then finish last (measured at
+    // 16 rows). One CTA, or a grid that fills the device (where the next kernel is a tensor-core linear whose
+    // set-up then overlaps this kernel's tail), release their dependents at once.
+    if (M <= R4K_ROWS || M > PDL_MAX_ROWS) pdl_launch_dependents();
     pdl_wait();   // x may be the output of the kernel before this one
     const int g = threadIdx.x >> 6, u = threadIdx.x & 63;  // row group, thread within the row
     float* buf = reinterpret_cast<float*>(smem_raw) + g * R4K;
@@ -545,12 +543,8 @@ static void launch_rotate(const __half* x, int M, int K, int64_t ldx, const int3
         if (setup.run([](int*) { return set_max_dynamic_smem(quantize_rows_rotate_kernel<E, SINK>, (32 + 16384) * 4); }) != SQAP_OK)
             return;
     }
-    if (M <= PDL_MAX_ROWS) {
-        const cudaError_t e = launch_dependent(quantize_rows_rotate_kernel<E, SINK>, dim3(M), dim3(T), smem, s, x, K, ldx, row_index, norm, o);
-        if (e != cudaSuccess) note_cuda_error(e);
-        return;
-    }
-    quantize_rows_rotate_kernel<E, SINK><<<M, T, smem, s>>>(x, K, ldx, row_index, norm, o);
+    const cudaError_t e = launch_dependent(quantize_rows_rotate_kernel<E, SINK>, dim3(M), dim3(T), smem, s, x, K, ldx, row_index, norm, o);
+    if (e != cudaSuccess) note_cuda_error(e);
 }
 
 template <int SINK>
@@ -564,13 +558,9 @@ static sqap_status launch_quantize(const __half* x, int M, int K, int64_t ldx, c
             int ctas = (M + R4K_ROWS - 1) / R4K_ROWS;
             const int resident = 2 * sm_count();
             if (ctas > resident) ctas = resident;
-            if (M <= PDL_MAX_ROWS) {
-                const cudaError_t e = launch_dependent(quantize_rotate4096_kernel<SINK>, dim3(ctas), dim3(R4K_THREADS), R4K_SMEM, s,
-                                                       x, M, ldx, row_index, o);
-                if (e != cudaSuccess) note_cuda_error(e);
-            } else {
-                quantize_rotate4096_kernel<SINK><<<ctas, R4K_THREADS, R4K_SMEM, s>>>(x, M, ldx, row_index, o);
-            }
+            const cudaError_t e = launch_dependent(quantize_rotate4096_kernel<SINK>, dim3(ctas), dim3(R4K_THREADS), R4K_SMEM, s,
+                                                   x, M, ldx, row_index, o);
+            if (e != cudaSuccess) note_cuda_error(e);
         }
         // E elements per thread: 16 from K = 512 up (T = K/16 <= 1024), fewer for short rows so a full warp works
         else if (K >= 512) launch_rotate<16, SINK>(x, M, K, ldx, row_index, o, s);

@@ -308,38 +308,45 @@ __device__ __forceinline__ void bar_sync_named(int id, int nthreads) {
     asm volatile("bar.sync %0, %1;" ::"r"(id), "r"(nthreads) : "memory");
 }
 
-// v: the raw sums of this thread's channel for 16 consecutive tokens starting at token m_first of the matrix.
-// ch: the thread's channel within the tile (plain: 0..127 = tensor-memory lane; SwiGLU: 0..63, gate and up of a
-// channel sit 16 lanes apart); n_tile0: first output channel of the tile; sw: this lane's weight scale.
-// stage: the buffer for this chunk; tid_half: 0..127 among the threads sharing it; bar_id: their named barrier.
-template <int OUT, bool SWIGLU>
-__device__ __forceinline__ void epilogue_chunk_coalesced(const Args& a, const uint32_t* v, int m_first, int n_tile0, int ch,
-                                                         float sw, int lane, const int4* t4, uint8_t* stage, int tid_half,
-                                                         int bar_id) {
+template <int OUT>
+__device__ __forceinline__ uint16_t bits16(float y) {
     static_assert(OUT == SQAP_FP16 || OUT == SQAP_BF16, "16-bit outputs only");
-    constexpr int ROWB = SWIGLU ? 128 : 256;   // bytes of one token's channels in the buffer
-    auto bits16 = [](float y) -> uint16_t {
-        return OUT == SQAP_FP16 ? __half_as_ushort(__float2half_rn(y)) : __bfloat16_as_ushort(__float2bfloat16_rn(y));
-    };
-    const bool odd = (lane & 16) != 0;         // SwiGLU: this lane holds the up projection, lane ^ 16 the gate
-    uint8_t* mine = stage + ch * 2;
-#pragma unroll
-    for (int j = 0; j < 16; j += 2) {
-        const int4 t = t4[j >> 1];
-        const int t0 = (static_cast<int>(v[j]) - t.x) >> 4, t1 = (static_cast<int>(v[j + 1]) - t.z) >> 4;
-        const float y0 = __fmul_rn(__fmul_rn(static_cast<float>(t0), __int_as_float(t.y)), sw);
-        const float y1 = __fmul_rn(__fmul_rn(static_cast<float>(t1), __int_as_float(t.w)), sw);
-        if (SWIGLU) {
-            // the gate lane finishes token j (needs the up value of its partner), the up lane token j+1
-            const float got = __shfl_xor_sync(0xffffffffu, odd ? y0 : y1, 16);
-            const float h = odd ? silu_mul_fast(got, y1) : silu_mul_fast(y0, got);
-            *reinterpret_cast<uint16_t*>(mine + (odd ? j + 1 : j) * ROWB) = bits16(h);
-        } else {
-            *reinterpret_cast<uint16_t*>(mine + j * ROWB) = bits16(y0);
-            *reinterpret_cast<uint16_t*>(mine + (j + 1) * ROWB) = bits16(y1);
-        }
+    return OUT == SQAP_FP16 ? __half_as_ushort(__float2half_rn(y)) : __bfloat16_as_ushort(__float2bfloat16_rn(y));
+}
+
+// Four consecutive tokens of this thread's channel: raw sums v0..v3 -> 16-bit outputs in the staging buffer.
+// tq: the four tokens' constants (two int4, see epilogue_chunk); mine: the buffer position of the first of the four
+// tokens for this thread's channel; ROWB apart per token. SwiGLU: gate and up of a channel sit 16 lanes apart; the
+// gate lane finishes tokens 0 and 2 (it needs the up value of its partner), the up lane tokens 1 and 3.
+template <int OUT, bool SWIGLU>
+__device__ __forceinline__ void epilogue_quad_to_stage(uint32_t v0, uint32_t v1, uint32_t v2, uint32_t v3, const int4* tq,
+                                                       float sw, bool odd, uint8_t* mine) {
+    constexpr int ROWB = SWIGLU ? 128 : 256;
+    const int4 ta = tq[0], tb = tq[1];
+    const float y0 = __fmul_rn(__fmul_rn(static_cast<float>((static_cast<int>(v0) - ta.x) >> 4), __int_as_float(ta.y)), sw);
+    const float y1 = __fmul_rn(__fmul_rn(static_cast<float>((static_cast<int>(v1) - ta.z) >> 4), __int_as_float(ta.w)), sw);
+    const float y2 = __fmul_rn(__fmul_rn(static_cast<float>((static_cast<int>(v2) - tb.x) >> 4), __int_as_float(tb.y)), sw);
+    const float y3 = __fmul_rn(__fmul_rn(static_cast<float>((static_cast<int>(v3) - tb.z) >> 4), __int_as_float(tb.w)), sw);
+    if (SWIGLU) {
+        const float g0 = __shfl_xor_sync(0xffffffffu, odd ? y0 : y1, 16);
+        const float g1 = __shfl_xor_sync(0xffffffffu, odd ? y2 : y3, 16);
+        const float h0 = odd ? silu_mul_fast(g0, y1) : silu_mul_fast(y0, g0);
+        const float h1 = odd ? silu_mul_fast(g1, y3) : silu_mul_fast(y2, g1);
+        *reinterpret_cast<uint16_t*>(mine + (odd ? 1 : 0) * ROWB) = bits16<OUT>(h0);
+        *reinterpret_cast<uint16_t*>(mine + (odd ? 3 : 2) * ROWB) = bits16<OUT>(h1);
+    } else {
+        *reinterpret_cast<uint16_t*>(mine) = bits16<OUT>(y0);
+        *reinterpret_cast<uint16_t*>(mine + ROWB) = bits16<OUT>(y1);
+        *reinterpret_cast<uint16_t*>(mine + 2 * ROWB) = bits16<OUT>(y2);
+        *reinterpret_cast<uint16_t*>(mine + 3 * ROWB) = bits16<OUT>(y3);
     }
-    bar_sync_named(bar_id, 128);
+}
+
+// A staged chunk ([16 tokens][64 or 128 channels] of 16-bit outputs) -> global memory, 16 bytes per thread.
+template <bool SWIGLU>
+__device__ __forceinline__ void epilogue_stage_copy_out(const Args& a, int m_first, int n_tile0, const uint8_t* stage,
+                                                        int tid_half) {
+    constexpr int ROWB = SWIGLU ? 128 : 256;
     constexpr int PPR = ROWB / 16;             // 16-byte pieces (8 channels) per token
 #pragma unroll
     for (int p = tid_half; p < 16 * PPR; p += 128) {
@@ -356,6 +363,25 @@ __device__ __forceinline__ void epilogue_chunk_coalesced(const Args& a, const ui
             }
         }
     }
+}
+
+// v: the raw sums of this thread's channel for 16 consecutive tokens starting at token m_first of the matrix.
+// ch: the thread's channel within the tile (plain: 0..127 = tensor-memory lane; SwiGLU: 0..63, gate and up of a
+// channel sit 16 lanes apart); n_tile0: first output channel of the tile; sw: this lane's weight scale.
+// stage: the buffer for this chunk; tid_half: 0..127 among the threads sharing it; bar_id: their named barrier.
+template <int OUT, bool SWIGLU>
+__device__ __forceinline__ void epilogue_chunk_coalesced(const Args& a, const uint32_t* v, int m_first, int n_tile0, int ch,
+                                                         float sw, int lane, const int4* t4, uint8_t* stage, int tid_half,
+                                                         int bar_id) {
+    constexpr int ROWB = SWIGLU ? 128 : 256;   // bytes of one token's channels in the buffer
+    const bool odd = (lane & 16) != 0;         // SwiGLU: this lane holds the up projection, lane ^ 16 the gate
+    uint8_t* mine = stage + ch * 2;
+#pragma unroll
+    for (int q = 0; q < 4; ++q)
+        epilogue_quad_to_stage<OUT, SWIGLU>(v[4 * q], v[4 * q + 1], v[4 * q + 2], v[4 * q + 3], t4 + 2 * q, sw, odd,
+                                            mine + 4 * q * ROWB);
+    bar_sync_named(bar_id, 128);
+    epilogue_stage_copy_out<SWIGLU>(a, m_first, n_tile0, stage, tid_half);
 }
 
 // Tokens [c_begin, c_end) of a finished accumulator tile through the routine above. stage_half: this half's two
