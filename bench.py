@@ -4,7 +4,8 @@ observations, with the quantization-aware visual-token pruning between two layer
 
 One step (per rank, 16 observations x 288 token rows = 4608 rows, configuration 4 of the workload):
   layer A at M = 4608 : quantize(+Hadamard) -> QKV -> quantize -> O -> quantize -> gate/up (SwiGLU) -> quantize -> down
-  prune               : scores -> top-k U ring U FPS -> compaction -> row gather   (256 -> 128 visual tokens)
+  prune               : scores -> top-k U ring U FPS -> compaction (256 -> 128 visual tokens); the kept rows leave
+                        as a source-row list, so the gather is folded into layer B's first quantizer
   layer B at M = 2560 : the same four linears on the surviving rows (distinct weights)
   decode              : one new token per observation (M = 16) through layer B's linears
 `value` = algorithmic tera-ops (2*M*N*K of every linear) per second of whole-step time, all ranks.
@@ -157,10 +158,11 @@ class Path:
         self.o = t.empty(M, wl.HIDDEN, dtype=f16, device=device)
         self.h = t.empty(M, wl.FFN, dtype=f16, device=device)
         self.d = t.empty(M, wl.HIDDEN, dtype=f16, device=device)
-        self.x1 = t.empty(M_PRUNED, wl.HIDDEN, dtype=f16, device=device)
+        self.x1 = t.empty(M_PRUNED, wl.HIDDEN, dtype=f16, device=device)   # only for timing the gather kernel alone
         self.d1 = t.empty(M_PRUNED, wl.HIDDEN, dtype=f16, device=device)
         self.ddec = t.empty(N_OBS, wl.HIDDEN, dtype=f16, device=device)
         self.kept = t.empty(N_OBS, wl.ROWS, dtype=i32, device=device)
+        self.row_index = t.empty(M_PRUNED, dtype=i32, device=device)
         self.nkept = t.empty(N_OBS, dtype=i32, device=device)
         self.ws_bytes = B.sqap_quantize_linear_workspace_bytes(M, wl.QKV, wl.FFN)
         self.ws = t.empty(self.ws_bytes, dtype=u8, device=device)
@@ -180,14 +182,14 @@ class Path:
                         kept=self.kept)]
         self.io.append({k: t.empty_like(v) for k, v in self.io[0].items()})
 
-    def linear(self, x_ptr, M, K, ldx, w, w_up, out, rotate=False, flags=0):
+    def linear(self, x_ptr, M, K, ldx, w, w_up, out, rotate=False, flags=0, row_index=None):
         B = self.B
-        B.sqap_quantize_linear(x_ptr, M, ldx, None, B.SQAP_Q_ROTATE if rotate else 0, w, w_up, out, out.shape[1],
+        B.sqap_quantize_linear(x_ptr, M, ldx, row_index, B.SQAP_Q_ROTATE if rotate else 0, w, w_up, out, out.shape[1],
                                B.SQAP_FP16, flags, self.ws, self.ws_bytes)
 
-    def layer(self, x, M, L: Layer, d_out):
+    def layer(self, x, M, L: Layer, d_out, row_index=None):
         H = wl.HIDDEN
-        self.linear(x.data_ptr(), M, H, H, L.w["qkv"], None, self.qkv, rotate=True)
+        self.linear(x.data_ptr(), M, H, H, L.w["qkv"], None, self.qkv, rotate=True, row_index=row_index)
         self.linear(self.qkv.data_ptr() + 2 * 2 * H, M, H, wl.QKV, L.w["o"], None, self.o)   # V third of QKV
         self.linear(self.o.data_ptr(), M, H, H, L.w["gate"], L.w["up"], self.h)
         self.linear(self.h.data_ptr(), M, wl.FFN, wl.FFN, L.w["down"], None, d_out)
@@ -195,9 +197,10 @@ class Path:
     def step(self, k: int = 0):
         B, io = self.B, self.io[k]
         self.layer(io["x"], M_FULL, self.layers[0], self.d)
-        B.sqap_prune_tokens(self.prune_params, io["scores"], io["centers"], io["x"], wl.HIDDEN, wl.HIDDEN, self.x1,
-                            wl.HIDDEN, ROWS_KEPT, io["kept"], self.nkept)
-        self.layer(self.x1, M_PRUNED, self.layers[1], io["d1"])
+        # the criterion writes the kept rows as a source-row list; layer B's first quantizer reads them in place
+        B.sqap_prune_select(self.prune_params, io["scores"], io["centers"], ROWS_KEPT, io["kept"], self.nkept,
+                            self.row_index)
+        self.layer(io["x"], M_PRUNED, self.layers[1], io["d1"], row_index=self.row_index)
         self.layer(io["xdec"], N_OBS, self.layers[1], io["ddec"])
 
     def upload(self, k: int = 0):
@@ -238,7 +241,7 @@ def _within_tolerance(got_bits, ref_bits):
 
 def check_step_against_oracle(torch, path: Path, step_fn):
     """Untimed. Replays the timed step once more and compares what it left on the device with the CPU oracle:
-    the kept-token indices of every observation (bit-exact), the gathered rows (bit-exact), and, for sampled token
+    the kept-token indices of every observation and their source-row list (bit-exact), and, for sampled token
     rows of the pruned layer and of the decode step, every linear of the chain on the input it actually received
     (the oracle applied to the device's own input of that stage), fp16 within max(1 ulp, 2e-3)."""
     import oracle
@@ -252,9 +255,10 @@ def check_step_against_oracle(torch, path: Path, step_fn):
     kept_o, nk_o = oracle.prune_tokens(path.prune_params, bits(inp["scores"]), inp["centers"])
     if not (np.array_equal(kept, kept_o) and np.array_equal(path.nkept.cpu().numpy(), nk_o)):
         return False, "kept indices differ from the oracle"
+    want_rows = (np.arange(N_OBS)[:, None] * wl.ROWS + kept_o[:, :ROWS_KEPT]).reshape(-1)
+    if not ((nk_o == ROWS_KEPT).all() and np.array_equal(path.row_index.cpu().numpy(), want_rows)):
+        return False, "the kept rows' source-row list differs from the oracle"
     x1_o = oracle.gather_rows(bits(inp["x"]), kept_o, nk_o, ROWS_KEPT).reshape(M_PRUNED, wl.HIDDEN)
-    if not np.array_equal(bits(path.x1.cpu().numpy()), x1_o):
-        return False, "gathered rows differ from the oracle"
 
     def lin(x_bits, name, rotate=False, up=None):
         _, s, codes = oracle.quantize_act(np.ascontiguousarray(x_bits), rotate=rotate)
@@ -279,7 +283,7 @@ def check_step_against_oracle(torch, path: Path, step_fn):
             ok = _within_tolerance(got, ref)
             if not ok.all():
                 return False, f"{what}, {name}: {int((~ok).sum())} of {ok.size} sampled outputs outside tolerance"
-    return True, (f"kept indices and gathered rows of {N_OBS} observations bit-exact; {len(rows_b)} rows of the pruned layer and "
+    return True, (f"kept indices and source-row list of {N_OBS} observations bit-exact; {len(rows_b)} rows of the pruned layer and "
                   f"{len(rows_d)} decode rows through all four linears within max(1 ulp, 2e-3) of the oracle")
 
 

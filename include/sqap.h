@@ -251,6 +251,19 @@ sqap_status sqap_prune_tokens(const sqap_prune_params* p, const void* scores, co
                               int32_t* kept_idx, int32_t* n_kept, void* stream);
 
 /*
+ * The same criterion and compaction without the row copy (the paper only needs the reduced sequence to reach the next
+ * layer; Section 4.3's speed-up is end to end, so a pass over the activations that can be avoided is avoided):
+ * besides kept_idx / n_kept as above, writes the kept rows as SOURCE ROW NUMBERS of the whole batch,
+ *   row_index[b*out_rows + i] = b*rows + kept_idx[b][i]      for i < min(n_kept[b], out_rows),
+ * which sqap_quantize_act / sqap_quantize_linear take as their `row_index` with M = batch*out_rows: the first linear
+ * after the pruning then reads the surviving rows where they are. Entries from n_kept[b] on (only when fewer rows
+ * were kept than out_rows) repeat the observation's last kept row, so every entry names an existing row.
+ * row_index: device int32 [batch*out_rows]; batch*rows must fit int32. Errors: as sqap_prune_tokens.
+ */
+sqap_status sqap_prune_select(const sqap_prune_params* p, const void* scores, const int32_t* ring_center, int out_rows,
+                              int32_t* kept_idx, int32_t* n_kept, int32_t* row_index, void* stream);
+
+/*
  * Attention scores of one task-query token over the visual tokens (strategy 1 of Section "Quantization-aware
  * Pruning Strategies" scores the visual tokens by the attention of a task-query token), computed from the fp16
  * output of a fused QKV projection. For observation b, head h and visual token j:

@@ -29,7 +29,7 @@ def SQAP_L_KSPLIT(n: int) -> int:
 EXPORTS = ("sqap_pack_weights", "sqap_quantize_weights", "sqap_free_weights", "sqap_weights_info", "sqap_unpack_weights",
            "sqap_quantize_act", "sqap_quantize_act_ex", "sqap_workspace_bytes", "sqap_w4a4_linear", "sqap_w4a4_linear_static",
            "sqap_quantize_linear", "sqap_quantize_linear_workspace_bytes",
-           "sqap_prune_tokens", "sqap_attention_scores",
+           "sqap_prune_tokens", "sqap_prune_select", "sqap_attention_scores",
            "sqap_project_center", "sqap_device_status", "sqap_last_cuda_error", "sqap_status_string",
            "sqap_kernel_launch_count", "sqap_selftest_bounded_wait")
 
@@ -76,6 +76,7 @@ def lib() -> ctypes.CDLL:
     L.sqap_quantize_linear_workspace_bytes.restype = sz
     L.sqap_quantize_linear.argtypes = [vp, i32, i64, vp, u32, vp, vp, vp, i64, i32, u32, vp, sz, vp]
     L.sqap_prune_tokens.argtypes = [ctypes.POINTER(PruneParams), vp, vp, vp, i64, i32, vp, i64, i32, vp, vp, vp]
+    L.sqap_prune_select.argtypes = [ctypes.POINTER(PruneParams), vp, vp, i32, vp, vp, vp, vp]
     L.sqap_attention_scores.argtypes = [vp, i64, i32, i32, i32, i32, i32, i32, i32, i32, i32, vp, vp]
     L.sqap_project_center.argtypes = [ctypes.POINTER(ctypes.c_double)] * 3 + [ctypes.c_double, ctypes.c_double,
                                                                               ctypes.POINTER(ctypes.c_int32),
@@ -218,6 +219,13 @@ def sqap_prune_tokens(params: dict, scores, ring_center, x, ldx: int, K: int, x_
     _check(lib().sqap_prune_tokens(ctypes.byref(p), _ptr(scores), _ptr(ring_center), _ptr(x), ldx, K, _ptr(x_out),
                                    ldo, out_rows, _ptr(kept_idx), _ptr(n_kept), _stream(stream)),
            "sqap_prune_tokens")
+
+
+def sqap_prune_select(params: dict, scores, ring_center, out_rows: int, kept_idx, n_kept, row_index, stream=None):
+    """The criterion without the row copy: kept indices plus the flat source-row list for a quantizer's row_index."""
+    p = PruneParams(**{k: int(v) for k, v in params.items()})
+    _check(lib().sqap_prune_select(ctypes.byref(p), _ptr(scores), _ptr(ring_center), out_rows, _ptr(kept_idx),
+                                   _ptr(n_kept), _ptr(row_index), _stream(stream)), "sqap_prune_select")
 
 
 def sqap_attention_scores(qkv, ldq: int, batch: int, rows: int, query_row: int, visual_start: int, n_visual: int,

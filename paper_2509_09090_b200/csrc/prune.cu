@@ -15,7 +15,8 @@ template <int CAND>
 __global__ void __launch_bounds__(512) prune_select_kernel(sqap_prune_params p, const void* __restrict__ scores,
                                                             const int32_t* __restrict__ ring_center,
                                                             int32_t* __restrict__ kept_idx,
-                                                            int32_t* __restrict__ n_kept) {
+                                                            int32_t* __restrict__ n_kept,
+                                                            int32_t* __restrict__ row_index, int out_rows) {
     __shared__ float a[PRUNE_MAX_VISUAL];
     __shared__ uint8_t keep[PRUNE_MAX_VISUAL];  // bit 0: in K_attn U K_ring, bit 1: in K_fps
     __shared__ int warp_tot[32];
@@ -132,12 +133,23 @@ __global__ void __launch_bounds__(512) prune_select_kernel(sqap_prune_params p, 
             before += (w < warp) ? t : 0;
             total += t;
         }
-        if (k) out[base + before + __popc(bal & ((1u << lane) - 1u))] = r;
+        if (k) {
+            const int pos = base + before + __popc(bal & ((1u << lane) - 1u));
+            out[pos] = r;
+            // the same list as source rows of the whole batch, for a quantizer that reads the kept rows in place
+            if (row_index && pos < out_rows) row_index[static_cast<int64_t>(b) * out_rows + pos] = b * p.rows + r;
+        }
         base += total;
         __syncthreads();
     }
     for (int r = base + tid; r < p.rows; r += blockDim.x) out[r] = -1;
     if (tid == 0) n_kept[b] = base;
+    if (row_index) {
+        // entries past n_kept repeat the observation's last kept row (its first row if nothing was kept), so that
+        // every entry names a row that exists
+        const int pad = b * p.rows + (base > 0 ? out[base - 1] : 0);   // written before the last __syncthreads
+        for (int i = base + tid; i < out_rows; i += blockDim.x) row_index[static_cast<int64_t>(b) * out_rows + i] = pad;
+    }
 }
 
 // Row copy: grid (out_rows, batch); CTA (i, b) copies row kept_idx[b][i] of observation b.
@@ -251,10 +263,9 @@ extern "C" sqap_status sqap_attention_scores(const void* qkv, int64_t ldq, int b
     return check_launch();
 }
 
-extern "C" sqap_status sqap_prune_tokens(const sqap_prune_params* p, const void* scores, const int32_t* ring_center,
-                                         const void* x, int64_t ldx, int K, void* x_out, int64_t ldo, int out_rows,
-                                         int32_t* kept_idx, int32_t* n_kept, void* stream) {
-    using namespace sqap;
+namespace sqap {
+
+static sqap_status prune_check(const sqap_prune_params* p, const void* scores, const int32_t* kept_idx, const int32_t* n_kept) {
     if (!p) return SQAP_ERR_INVALID;
     if (p->batch < 0 || p->rows < 0 || p->n_visual < 0 || p->visual_start < 0 ||
         static_cast<int64_t>(p->visual_start) + p->n_visual > p->rows)
@@ -267,24 +278,54 @@ extern "C" sqap_status sqap_prune_tokens(const sqap_prune_params* p, const void*
     if (p->batch > 65535) return SQAP_ERR_UNSUPPORTED;
     if (p->batch == 0) return SQAP_OK;
     if (!kept_idx || !n_kept || (p->n_visual > 0 && !scores)) return SQAP_ERR_INVALID;
-    if (x) {
-        if (!x_out || K <= 0 || ldx < K || ldo < K || out_rows < 0) return SQAP_ERR_INVALID;
-        if (K % 8 != 0 || ldx % 8 != 0 || ldo % 8 != 0 || !aligned16(x) || !aligned16(x_out)) return SQAP_ERR_ALIGN;
-    }
-    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    return SQAP_OK;
+}
+
+static sqap_status launch_select(const sqap_prune_params* p, const void* scores, const int32_t* ring_center,
+                                 int32_t* kept_idx, int32_t* n_kept, int32_t* row_index, int out_rows, cudaStream_t s) {
     sqap_prune_params q = *p;
     if (q.n_visual == 0) q.grid_w = q.grid_h = 1;
     int threads = (q.n_visual + 31) / 32 * 32;
     if (threads < 128) threads = 128;
     if (threads > 512) threads = 512;
-    if (q.n_visual <= 256) prune_select_kernel<8><<<q.batch, threads, 0, s>>>(q, scores, ring_center, kept_idx, n_kept);
-    else prune_select_kernel<32><<<q.batch, threads, 0, s>>>(q, scores, ring_center, kept_idx, n_kept);
+    if (q.n_visual <= 256)
+        prune_select_kernel<8><<<q.batch, threads, 0, s>>>(q, scores, ring_center, kept_idx, n_kept, row_index, out_rows);
+    else
+        prune_select_kernel<32><<<q.batch, threads, 0, s>>>(q, scores, ring_center, kept_idx, n_kept, row_index, out_rows);
     count_launch();
-    sqap_status st = check_launch();
+    return check_launch();
+}
+
+}  // namespace sqap
+
+extern "C" sqap_status sqap_prune_select(const sqap_prune_params* p, const void* scores, const int32_t* ring_center,
+                                         int out_rows, int32_t* kept_idx, int32_t* n_kept, int32_t* row_index,
+                                         void* stream) {
+    using namespace sqap;
+    const sqap_status st = prune_check(p, scores, kept_idx, n_kept);
+    if (st != SQAP_OK || p->batch == 0) return st;
+    if (out_rows < 0 || (out_rows > 0 && !row_index)) return SQAP_ERR_INVALID;
+    if (static_cast<int64_t>(p->batch) * p->rows > 0x7FFFFFFFll) return SQAP_ERR_UNSUPPORTED;   // row numbers are int32
+    return launch_select(p, scores, ring_center, kept_idx, n_kept, out_rows > 0 ? row_index : nullptr, out_rows,
+                         static_cast<cudaStream_t>(stream));
+}
+
+extern "C" sqap_status sqap_prune_tokens(const sqap_prune_params* p, const void* scores, const int32_t* ring_center,
+                                         const void* x, int64_t ldx, int K, void* x_out, int64_t ldo, int out_rows,
+                                         int32_t* kept_idx, int32_t* n_kept, void* stream) {
+    using namespace sqap;
+    sqap_status st = prune_check(p, scores, kept_idx, n_kept);
+    if (st != SQAP_OK || p->batch == 0) return st;
+    if (x) {
+        if (!x_out || K <= 0 || ldx < K || ldo < K || out_rows < 0) return SQAP_ERR_INVALID;
+        if (K % 8 != 0 || ldx % 8 != 0 || ldo % 8 != 0 || !aligned16(x) || !aligned16(x_out)) return SQAP_ERR_ALIGN;
+    }
+    cudaStream_t s = static_cast<cudaStream_t>(stream);
+    st = launch_select(p, scores, ring_center, kept_idx, n_kept, nullptr, 0, s);
     if (st != SQAP_OK) return st;
     if (x && out_rows > 0) {
-        dim3 grid(out_rows, q.batch);
-        gather_rows_kernel<<<grid, 256, 0, s>>>(static_cast<const __half*>(x), ldx, q.rows, K, kept_idx, n_kept,
+        dim3 grid(out_rows, p->batch);
+        gather_rows_kernel<<<grid, 256, 0, s>>>(static_cast<const __half*>(x), ldx, p->rows, K, kept_idx, n_kept,
                                                 static_cast<__half*>(x_out), ldo, out_rows);
         count_launch();
         st = check_launch();

@@ -35,7 +35,7 @@ class Stack:
         self.o_dec = t.empty(nd, 1, H, dtype=f16, device=device)
         self.h_dec = t.empty(nd, 1, F, dtype=f16, device=device)
         self.d_dec = t.empty(n_decode, nl, 1, H, dtype=f16, device=device)
-        self.x1 = t.empty(self.rows_kept, H, dtype=f16, device=device)
+        self.row_index = t.empty(self.rows_kept, dtype=i32, device=device)   # the kept rows, as source rows of x
         self.kept = t.empty(1, rows, dtype=i32, device=device)
         self.nkept = t.empty(1, dtype=i32, device=device)
         self.prune_params = wl.prune_params(1, rows, wl.VISUAL_START, wl.N_VISUAL, wl.GRID, wl.GRID, 32, k_attn, keep,
@@ -44,29 +44,30 @@ class Stack:
         self.ws = t.empty(self.ws_bytes, dtype=t.uint8, device=device)
         self.keep_intermediates = keep_intermediates
 
-    def _lin(self, x_ptr, m, ldx, w, w_up, out, rotate=False):
+    def _lin(self, x_ptr, m, ldx, w, w_up, out, rotate=False, row_index=None):
         B = self.B
-        B.sqap_quantize_linear(x_ptr, m, ldx, None, B.SQAP_Q_ROTATE if rotate else 0, w, w_up, out, out.shape[-1],
+        B.sqap_quantize_linear(x_ptr, m, ldx, row_index, B.SQAP_Q_ROTATE if rotate else 0, w, w_up, out, out.shape[-1],
                                B.SQAP_FP16, 0, self.ws, self.ws_bytes)
 
-    def _layer(self, x, m, L, qkv, o, h, d):
+    def _layer(self, x, m, L, qkv, o, h, d, row_index=None):
         H = wl.HIDDEN
-        self._lin(x.data_ptr(), m, H, L["qkv"], None, qkv, rotate=True)
+        self._lin(x.data_ptr(), m, H, L["qkv"], None, qkv, rotate=True, row_index=row_index)
         self._lin(qkv.data_ptr() + 2 * 2 * H, m, wl.QKV, L["o"], None, o)      # the V third of the fused output
         self._lin(o.data_ptr(), m, H, L["gate"], L["up"], h)
         self._lin(h.data_ptr(), m, wl.FFN, L["down"], None, d)
 
     def prefill(self, x, scores, centers):
-        """x: fp16 [rows, HIDDEN]; scores: fp16 [1, 32, N_VISUAL]; centers: int32 [1, 2] (device tensors)."""
-        H = wl.HIDDEN
+        """x: fp16 [rows, HIDDEN]; scores: fp16 [1, 32, N_VISUAL]; centers: int32 [1, 2] (device tensors).
+        From the prune layer on, the first linear of a layer reads the surviving rows of x in place, through the row
+        list the criterion wrote (no gathered copy is made)."""
         for li, L in enumerate(self.layers):
             if li == self.prune_after:
-                self.B.sqap_prune_tokens(self.prune_params, scores, centers, x, H, H, self.x1, H, self.rows_kept,
-                                         self.kept, self.nkept)
+                self.B.sqap_prune_select(self.prune_params, scores, centers, self.rows_kept, self.kept, self.nkept,
+                                         self.row_index)
             pruned = li >= self.prune_after
             i = li if self.keep_intermediates else 0
-            self._layer(self.x1 if pruned else x, self.rows_kept if pruned else self.rows, L, self.qkv[i], self.o[i],
-                        self.h[i], self.d[li])
+            self._layer(x, self.rows_kept if pruned else self.rows, L, self.qkv[i], self.o[i], self.h[i], self.d[li],
+                        row_index=self.row_index if pruned else None)
 
     def decode(self, xdec):
         """xdec: fp16 [n_decode, HIDDEN]: one new token per step through every layer."""

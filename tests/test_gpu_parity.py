@@ -608,6 +608,39 @@ def test_prune_fps_on_one_token_wide_and_high_grids(grid_w, grid_h):
         check_prune(p, s, np.array([[0, grid_h // 2], [grid_w - 1, 0]], np.int32))
 
 
+def test_prune_select_row_list_feeds_the_quantizer():
+    """sqap_prune_select: the same kept set as sqap_prune_tokens, and the flat source-row list b*rows + kept row (the
+    observation's last kept row repeated where fewer rows were kept than asked for); a quantize + linear that reads
+    x through that list equals one that reads the oracle's gathered copy."""
+    Bn, rows, K = 3, 70, 256
+    scores = wl.scores_normal(38, 1, Bn, 48)
+    centers = np.array([[2, 2], [7, 5], [30, 30]], np.int32)
+    x = wl.activations(38, 2, Bn * rows, K, 3, 20.0)
+    for keep, k_attn, radius, out_rows in [(24, 10, 1, 46), (24, 10, 1, 50), (0, 0, -1, 30)]:
+        p = wl.prune_params(Bn, rows, 5, 48, 8, 6, 0, k_attn, keep, ring_radius=radius)
+        kept_o, nk_o = oracle.prune_tokens(p, scores, centers)
+        kept = torch.full((Bn, rows), -7, dtype=torch.int32, device="cuda")
+        nk = torch.full((Bn,), -7, dtype=torch.int32, device="cuda")
+        ri = torch.full((Bn * out_rows + 1,), -7, dtype=torch.int32, device="cuda")
+        B.sqap_prune_select(p, G.to_dev(scores), G.to_dev(centers), out_rows, kept, nk, ri)
+        torch.cuda.synchronize()
+        assert np.array_equal(kept.cpu().numpy(), kept_o) and np.array_equal(nk.cpu().numpy(), nk_o)
+        want = np.empty((Bn, out_rows), np.int64)
+        for b in range(Bn):
+            n = min(int(nk_o[b]), out_rows)
+            want[b, :n] = b * rows + kept_o[b, :n]
+            want[b, n:] = b * rows + (kept_o[b, nk_o[b] - 1] if nk_o[b] > 0 else 0)
+        got = ri.cpu().numpy()
+        assert got[-1] == -7 and np.array_equal(got[:-1].reshape(Bn, out_rows), want)
+        wc, ws = wl.weight_codes(38, 3, 72, K), wl.weight_scales(38, 3, 72)
+        check_linear(x, wc, ws, rotate=True, row_index=want.reshape(-1).astype(np.int32), flags_list=[0])
+        w = G.pack(wc, ws)
+        a = G.quantize_linear(x, w, rotate=True, row_index=got[:-1])
+        b_ = G.quantize_linear(np.ascontiguousarray(x[want.reshape(-1)]), w, rotate=True)
+        assert np.array_equal(a, b_)
+        w.close()
+
+
 def test_prune_fps_worked_example():
     p = wl.prune_params(1, 256, 0, 256, 16, 16, 0, 0, 5)
     kept, nk, _ = G.prune(p, np.zeros((1, 256), np.float32))

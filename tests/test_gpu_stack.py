@@ -71,9 +71,10 @@ def test_config3_whole_stack_prefill_prune_decode_replayed_from_one_graph():
         st.prefill(x, scores, centers)      # eager once (first-call set-up happens outside the capture)
         st.decode(xdec)
         side.synchronize()
-        for buf in (st.qkv, st.o, st.h, st.d, st.qkv_dec, st.o_dec, st.h_dec, st.d_dec, st.x1):
+        for buf in (st.qkv, st.o, st.h, st.d, st.qkv_dec, st.o_dec, st.h_dec, st.d_dec):
             buf.view(torch.int16).fill_(0x7B7B)              # only what the replay writes may pass the check
         st.kept.fill_(-9)
+        st.row_index.fill_(-9)
         graph = torch.cuda.CUDAGraph()
         with torch.cuda.graph(graph, stream=side):
             st.prefill(x, scores, centers)
@@ -88,8 +89,9 @@ def test_config3_whole_stack_prefill_prune_decode_replayed_from_one_graph():
     kept_o, nk_o = oracle.prune_tokens(p, bits(inp["scores"]), centers_np)
     assert int(st.nkept.cpu()[0]) == int(nk_o[0]) == st.rows_kept
     assert np.array_equal(st.kept.cpu().numpy(), kept_o)
+    # the pruned layers read the kept rows of x in place: the row list must name exactly the oracle's kept rows
+    assert np.array_equal(st.row_index.cpu().numpy(), kept_o[0, :st.rows_kept])
     x1_o = oracle.gather_rows(bits(inp["x"])[None], kept_o, nk_o, st.rows_kept)[0]
-    assert np.array_equal(bits(st.x1.cpu().numpy()), x1_o)
 
     xd_bits = bits(inp["x_decode"])
     for li in range(n_layers):
