@@ -867,18 +867,25 @@ def run_single_kernel(args):
     if args.kernel == "quantize":
         for i in range(args.steps):
             B.sqap_quantize_act(x, M, H, H, None, B.SQAP_Q_ROTATE if i % 2 == 0 else 0, q, sx)
-    elif args.kernel in ("gemm", "gemv", "stream", "midm", "swiglu"):
-        names = {"gemm": ("qkv",), "gemv": ("qkv",), "stream": ("qkv",), "midm": ("o",), "swiglu": ("gate", "up")}[args.kernel]
+    elif args.kernel in ("gemm", "gemv", "stream", "midm", "downm", "swiglu"):
+        names = {"gemm": ("qkv",), "gemv": ("qkv",), "stream": ("qkv",), "midm": ("o",), "downm": ("down",),
+                 "swiglu": ("gate", "up")}[args.kernel]
         wts = wl.config4_weights(seed=4)
         ws = [B.sqap_pack_weights(np.ascontiguousarray(wts[n + "_codes"]), np.ascontiguousarray(wts[n + "_scales"]),
-                                  wts[n + "_codes"].shape[0], H) for n in names]
-        # stream: one decode token per observation; midm: one observation pruned to 160 rows (O projection)
-        Mk = {"gemv": 1, "stream": N_OBS, "midm": 160}.get(args.kernel, M)
+                                  wts[n + "_codes"].shape[0], wts[n + "_codes"].shape[1]) for n in names]
+        # stream: one decode token per observation; midm / downm: one observation pruned to 160 rows (O projection on
+        # the one-CTA-per-tile kernel; down projection, 11008 codes per row, on the cluster split-K kernel)
+        Mk = {"gemv": 1, "stream": N_OBS, "midm": 160, "downm": 160}.get(args.kernel, M)
         N = ws[0].N
+        Kk = ws[0].K
+        if Kk != H:
+            x = torch.from_numpy(wl.activations(4, 77, Mk, Kk, 110, 30.0)).to(dev)
+        H_ = H
+        H = Kk
         out = torch.empty(Mk, N, dtype=torch.float16, device=dev)
         nb = B.sqap_workspace_bytes(Mk, N, H)
         wsp = torch.empty(nb, dtype=torch.uint8, device=dev)
-        B.sqap_quantize_act(x, Mk, H, H, None, B.SQAP_Q_ROTATE, q, sx)
+        B.sqap_quantize_act(x, Mk, H, H, None, B.SQAP_Q_ROTATE if Kk == H_ else 0, q, sx)
         for i in range(args.steps):
             B.sqap_w4a4_linear(q, sx, Mk, ws[0], ws[1] if len(ws) > 1 else None, out, N, B.SQAP_FP16,
                                B.SQAP_L_REUSE_EXPANDED if i else 0, wsp, nb)
@@ -952,7 +959,7 @@ def main():
                     help="time every kernel of the path alone at the workload's shapes (one JSON table, no bench line)")
     ap.add_argument("--stack", action="store_true",
                     help="time configs[3] (32-layer stack: prefill + 7 decode tokens for one observation); own JSON line")
-    ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "stream", "midm", "quantize", "prune"],
+    ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "stream", "midm", "downm", "quantize", "prune"],
                     help="profiling aid: launch only this kernel --steps times (no bench line)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:

@@ -125,6 +125,13 @@ struct Weights {
     int N, K, half;      // half-block size of the nibble pairing (64 or 16)
     uint32_t flags;
     int device;
+    // Tensor maps of the packed matrix for the tensor-core kernels' TMA loads (rows of K/2 bytes, 128B swizzle, a box
+    // of 128 bytes x 128 rows, or x 64 rows where a gate / up pair shares a tile), encoded once at pack time: they
+    // depend on nothing but the handle. Opaque 128-byte CUtensorMap objects; has_maps = 0 where the kernels that use
+    // them cannot run the shape (K % 128 != 0) or the encoder is unavailable.
+    alignas(64) unsigned char map_rows128[128];
+    alignas(64) unsigned char map_rows64[128];
+    int has_maps;
 };
 
 }  // namespace sqap

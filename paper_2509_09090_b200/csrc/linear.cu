@@ -459,6 +459,8 @@ static LinearArgs make_args(void* workspace, const float* act_scales, int M, con
     a.w_scales = w->scales;
     a.w_up = w_up ? w_up->packed : nullptr;
     a.w_up_scales = w_up ? w_up->scales : nullptr;
+    a.w_handle = w;
+    a.w_up_handle = w_up;
     a.out = out;
     a.ldo = ldo;
     a.out_dtype = out_dtype;

@@ -18,6 +18,8 @@ struct LinearArgs {
     const __half* w_scales;
     const uint8_t* w_up;    // nullptr unless SwiGLU
     const __half* w_up_scales;
+    const Weights* w_handle;     // the handles themselves (for the tensor maps cached in them)
+    const Weights* w_up_handle;
     void* out;
     int64_t ldo;
     int out_dtype;

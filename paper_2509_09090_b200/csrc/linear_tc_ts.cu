@@ -375,10 +375,7 @@ sqap_status launch_linear_tcgen05_ts(const LinearArgs& a, cudaStream_t s) {
     if (!k.status) return SQAP_ERR_CUDA;
 
     CUtensorMap tm_w, tm_u, tm_x;
-    const uint32_t w_box_rows = k.swiglu ? BM / 2 : BM;
-    if (!make_map(&tm_w, a.w, a.N, a.K / 2, w_box_rows, BK / 2, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
-    if (!make_map(&tm_u, k.swiglu ? a.w_up : a.w, a.N, a.K / 2, w_box_rows, BK / 2, CU_TENSOR_MAP_SWIZZLE_128B))
-        return SQAP_ERR_CUDA;
+    if (!weight_maps(a, k.swiglu != 0, BM, BK / 2, &tm_w, &tm_u)) return SQAP_ERR_CUDA;
     if (!make_map(&tm_x, a.x8, a.M, a.K, k.BN, BKH, CU_TENSOR_MAP_SWIZZLE_128B)) return SQAP_ERR_CUDA;
 
     static PerDevice<int> setup;

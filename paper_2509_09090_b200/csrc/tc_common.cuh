@@ -4,6 +4,8 @@
 
 #include <cuda.h>
 
+#include <cstring>
+
 #include "linear.cuh"
 
 namespace sqap {
@@ -433,6 +435,36 @@ inline bool make_map(CUtensorMap* m, const void* ptr, uint64_t rows, uint64_t ro
     return fn(m, CU_TENSOR_MAP_DATA_TYPE_UINT8, 2, const_cast<void*>(ptr), dims, strides, box, estr,
               CU_TENSOR_MAP_INTERLEAVE_NONE, swz, CU_TENSOR_MAP_L2_PROMOTION_L2_256B,
               CU_TENSOR_MAP_FLOAT_OOB_FILL_NONE) == CUDA_SUCCESS;
+}
+
+// The two weight tensor maps of a launch (w and, for a gate / up pair, w_up; else w twice): taken from the handles
+// where they were encoded at pack time, encoded here otherwise. BKB = bytes of K per box row (128).
+inline bool weight_maps(const LinearArgs& a, bool swiglu, uint32_t rows_per_tile, uint32_t bkb, CUtensorMap* tm_w, CUtensorMap* tm_u) {
+    const uint32_t box_rows = swiglu ? rows_per_tile / 2 : rows_per_tile;
+    auto from_handle = [&](const Weights* h, CUtensorMap* out) {
+        if (!h || !h->has_maps || bkb != 128 || (box_rows != 128 && box_rows != 64)) return false;
+        memcpy(out, box_rows == 128 ? h->map_rows128 : h->map_rows64, sizeof(CUtensorMap));
+        return true;
+    };
+    if (!from_handle(a.w_handle, tm_w) && !make_map(tm_w, a.w, a.N, a.K / 2, box_rows, bkb, CU_TENSOR_MAP_SWIZZLE_128B)) return false;
+    if (!swiglu) {
+        *tm_u = *tm_w;
+        return true;
+    }
+    return from_handle(a.w_up_handle, tm_u) || make_map(tm_u, a.w_up, a.N, a.K / 2, box_rows, bkb, CU_TENSOR_MAP_SWIZZLE_128B);
+}
+
+// Encodes a handle's maps (weights.cu, at pack time).
+inline void encode_handle_maps(Weights* w) {
+    w->has_maps = 0;
+    if (w->half != 64) return;   // K % 128 != 0: the tensor-core kernels do not run the shape
+    static_assert(sizeof(CUtensorMap) == 128, "tensor map storage in the handle");
+    CUtensorMap a, b;
+    if (!make_map(&a, w->packed, w->N, w->K / 2, 128, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return;
+    if (!make_map(&b, w->packed, w->N, w->K / 2, 64, 128, CU_TENSOR_MAP_SWIZZLE_128B)) return;
+    memcpy(w->map_rows128, &a, 128);
+    memcpy(w->map_rows64, &b, 128);
+    w->has_maps = 1;
 }
 
 // Splits M tokens into m_tiles tiles of BN tokens (multiple of 16, <= bn_max) for a persistent kernel whose

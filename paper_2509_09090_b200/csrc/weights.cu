@@ -2,7 +2,7 @@
 // described in common.cuh, and its inverse for checking. Pure permutation / re-encoding.
 #include <new>
 
-#include "common.cuh"
+#include "tc_common.cuh"
 
 namespace sqap {
 
@@ -186,6 +186,7 @@ sqap_status sqap_pack_weights(const int8_t* codes, const uint16_t* scales_fp16, 
     }
     cudaFree(staged);
     cudaFree(bad);
+    tc::encode_handle_maps(w);
     *out = w;
     return SQAP_OK;
 fail:
