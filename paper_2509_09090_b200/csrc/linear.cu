@@ -503,11 +503,11 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
         const bool stream = mma_stream_supports(a) && !one_row_in_registers && (a.M <= 16 || w_tiles < 64);
         const bool gemv = !stream && a.M <= 8 && (!tc_ok || a.M <= 2 || (a.M <= 4 && w_tiles < 64));
         // CTA pairs fetch each token once per 256 weight rows: ahead from ~144 tokens on when there are enough pairs
-        const bool pairs = a.M >= 512 || (a.M >= 144 && w_tiles >= 64);
+        const bool pairs = a.M >= 512 || (a.M >= 144 && w_tiles >= 64) || (a.M > 320 && a.K >= 8192);
         // Few weight tiles and a long K (the down projection of one observation: 32 tiles x 43 stages): one cluster
         // per tile with K split over its CTAs; measured ahead of both other kernels there, behind them elsewhere
         // (its two cluster barriers and the exchange of partial sums cost about as much as 8 stages).
-        const bool split_k = !pairs && a.M >= 64 && w_tiles < 64 && a.K >= 8192;
+        const bool split_k = !pairs && a.M >= 64 && a.M <= 320 && w_tiles < 64 && a.K >= 8192;   // beyond ~320 rows the pairs win
         *path = stream ? PATH_MMA : gemv ? PATH_GEMV
                 : (tc_ok ? (pairs ? PATH_TC_PAIR : split_k ? PATH_TC_SPLITK : PATH_TC_TS) : PATH_SIMT);
     }

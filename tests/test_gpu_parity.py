@@ -372,11 +372,11 @@ def test_linear_register_mma_streamer(M, N, K, swiglu):
 @pytest.mark.parametrize("M,N,K,swiglu", [(1, 136, 4224, False), (16, 8192, 256, False), (17, 8192, 256, False),
                                           (32, 264, 384, True), (33, 264, 384, True), (143, 8192, 128, False),
                                           (144, 8192, 128, False), (150, 4096, 256, True), (63, 384, 8192, False),
-                                          (64, 384, 8192, False), (100, 384, 7936, False)])
+                                          (64, 384, 8192, False), (100, 384, 7936, False), (320, 384, 8192, False), (321, 384, 8192, False)])
 def test_linear_dispatch_boundaries(M, N, K, swiglu):
     """The kernel the dispatcher picks by itself on either side of each of its thresholds (one row longer than 4096
     codes; 16 | 17 rows with many weight tiles; 32 | 33 rows with few; 143 | 144 rows with many tiles, plain and
-    gated; few weight tiles with K below | from 8192 and 63 | 64 rows: the cluster split-K kernel), against the
+    gated; few weight tiles with K below | from 8192 and 63 | 64 and 320 | 321 rows: the cluster split-K kernel), against the
     oracle and against the plain CUDA-core kernel."""
     x = wl.activations(29, M + K, M, K, max(1, K // 100), 25.0)
     g = (wl.weight_codes(29, N + K, N, K), wl.weight_scales(29, N + K, N, mult=0.5))
