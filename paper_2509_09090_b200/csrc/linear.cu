@@ -238,21 +238,23 @@ __global__ void __launch_bounds__(256) w4a4_gemv_kernel(LinearArgs a) {
 // ---------------------------------------------------------------------------------------------
 // Single-row decode step (M = 1): the one activation row lives in registers. A lane always meets the same
 // 16-byte weight chunks (lane, lane + 32, ...) of whatever row its warp streams, so it loads the 2 x 16
-// activation bytes that go with each of them once and then only streams weights: two rows at a time (all their
-// loads issued before the first dp4a), persistent warps striding over the output channels.
+// activation bytes that go with each of them once and then only streams weights. An item is two weight rows (for a
+// gate / up pair: the same row of both matrices), all their loads issued before the first dp4a; for the gated pair a
+// warp keeps TWO items in flight in two register buffers and refills a buffer as soon as it has used it, so its
+// loads never stop while it computes. The first item(s) are fetched before the dependency wait. Persistent warps
+// stride over the output channels.
 // FUSEQ: the kernel also quantizes the row (plain per-token quantizer, no rotation): every CTA repeats the small
 // job (one 16-byte chunk or two per thread, two block-wide reductions) into shared memory while its first weight
 // rows are in flight, which takes a whole kernel out of a decode step's chain; CTA 0 also leaves the expanded codes,
 // their sum and the scale in the workspace, as the separate quantizer would have.
 template <bool SWIGLU, int CPL, bool FUSEQ>
-__global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
+__global__ void __launch_bounds__(256, SWIGLU ? 2 : 3) w4a4_gemv1_kernel(LinearArgs a) {
     __shared__ __align__(16) int8_t xs[FUSEQ ? 32 * 32 * CPL : 16];
     __shared__ float red_f[8];
     __shared__ int red_i[8];
     const int lane = threadIdx.x & 31;
     const int gw = blockIdx.x * (blockDim.x >> 5) + (threadIdx.x >> 5), W = gridDim.x * (blockDim.x >> 5);
     const int chunks = a.K / 32;
-    constexpr bool TWO = !SWIGLU;   // rows in flight per warp (the gated pair already streams two weight rows)
     auto load_row = [&](const uint8_t* wbase, int n, uint4* wv) {
         const uint4* row = reinterpret_cast<const uint4*>(wbase + static_cast<int64_t>(n) * (a.K / 2));
 #pragma unroll
@@ -261,15 +263,21 @@ __global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
             wv[i] = c < chunks ? __ldg(row + c) : make_uint4(0, 0, 0, 0);   // zero weights meet zero activations
         }
     };
-    auto load_rows = [&](int n, uint4* g0, uint4* g1, uint4* u0) {
-        load_row(a.w, n, g0);
-        if (SWIGLU) load_row(a.w_up, n, u0);
-        if (TWO && n + W < a.N) load_row(a.w, n + W, g1);
+    // item n: rows n and n + W of the matrix, or row n of the gate and of the up matrix
+    auto load_item = [&](int n, uint4* p, uint4* q) {
+        load_row(a.w, n, p);
+        if (SWIGLU) load_row(a.w_up, n, q);
+        else if (n + W < a.N) load_row(a.w, n + W, q);
     };
-    // The first rows' weights do not depend on the kernel before this one (the quantizer): fetch them, then wait.
-    // (Not for the gated pair: holding three rows across the wait costs the registers of the third resident CTA.)
-    uint4 g0[CPL], g1[TWO ? CPL : 1], u0[SWIGLU ? CPL : 1];
-    if (!SWIGLU && gw < a.N) load_rows(gw, g0, g1, u0);
+    const int step = (SWIGLU ? 1 : 2) * W;
+    // The first items' weights do not depend on the kernel before this one (the quantizer): fetch them, then wait.
+    // The gate / up pair (three to four items per warp at 11008 channels) runs two items deep: measured 11.5 -> 9.4 us.
+    // The plain matrices (one or two items per warp) gain nothing from the second buffer and lose the third resident
+    // CTA to its registers (QKV: 6.8 -> 7.1 us), so they keep one.
+    constexpr bool DEEP = SWIGLU;
+    uint4 A0[CPL], A1[CPL], B0[DEEP ? CPL : 1], B1[DEEP ? CPL : 1];
+    if (gw < a.N) load_item(gw, A0, A1);
+    if (DEEP && gw + step < a.N) load_item(gw + step, B0, B1);
     pdl_launch_dependents();
     pdl_wait();
     int bs;
@@ -378,18 +386,197 @@ __global__ void __launch_bounds__(256) w4a4_gemv1_kernel(LinearArgs a) {
         if (SWIGLU) y = swiglu(y, dequant(finish_acc(raw_u, bs), sx, __half2float(a.w_up_scales[n])));
         store_out(a.out, n, a.out_dtype, y, t);
     };
-    for (int n = gw; n < a.N; n += (TWO ? 2 : 1) * W) {
-        const int n2 = n + W;
-        const bool two = TWO && n2 < a.N;
-        if (SWIGLU || n != gw) load_rows(n, g0, g1, u0);
-        finish(n, dot(g0), SWIGLU ? dot(u0) : 0);
-        if (TWO && two) finish(n2, dot(g1), 0);
+    auto do_item = [&](int n, const uint4* p, const uint4* q) {
+        if (SWIGLU) {
+            finish(n, dot(p), dot(q));
+        } else {
+            finish(n, dot(p), 0);
+            if (n + W < a.N) finish(n + W, dot(q), 0);
+        }
+    };
+    if (DEEP) {
+        for (int n = gw; n < a.N; n += 2 * step) {
+            do_item(n, A0, A1);
+            if (n + 2 * step < a.N) load_item(n + 2 * step, A0, A1);
+            if (n + step < a.N) {
+                do_item(n + step, B0, B1);
+                if (n + 3 * step < a.N) load_item(n + 3 * step, B0, B1);
+            }
+        }
+    } else {
+        for (int n = gw; n < a.N; n += step) {
+            if (n != gw) load_item(n, A0, A1);
+            do_item(n, A0, A1);
+        }
     }
+}
+
+// ---------------------------------------------------------------------------------------------
+// Single-row decode step with a row longer than 4096 codes (the down projection: 11008): the activation codes do
+// not fit a lane's registers, so they live in shared memory, ordered the way the packed weight chunks meet them
+// (lo[c] / hi[c]: the 16 codes that meet the low / high nibbles of packed chunk c, so a warp's reads are contiguous).
+// A CTA owns a contiguous block of output channels (N / gridDim of them); its warps take the block's items (4096
+// codes = 2 KB of one weight row) round-robin, so that rows of two or three items spread over several warps and every
+// warp gets the same number of items to within one; two items are in flight per warp (two register buffers, used in
+// turn), both fetched before the dependency wait. The items' sums meet in shared memory, and the CTA finishes its
+// channels together at the end. FUSEQ as above (rows of up to
+// MMA_FUSE_MAX_K codes); otherwise the expanded codes come from the workspace.
+constexpr int GL_CPI = 4;   // 16-byte chunks per lane and item
+
+template <bool FUSEQ>
+__global__ void __launch_bounds__(256, 3) w4a4_gemv1_long_kernel(LinearArgs a) {
+    extern __shared__ __align__(16) uint8_t xs_long[];   // K bytes: lo array, then hi array
+    __shared__ float red_f[8];
+    __shared__ int red_i[8];
+    const int tid = threadIdx.x, lane = tid & 31, wid = tid >> 5;
+    const int chunks = a.K / 32, nseg = (chunks + 32 * GL_CPI - 1) / (32 * GL_CPI);
+    uint4* lo = reinterpret_cast<uint4*>(xs_long);
+    uint4* hi = reinterpret_cast<uint4*>(xs_long + a.K / 2);
+    auto load_item = [&](int n, int seg, uint4* wv) {
+        const uint4* row = reinterpret_cast<const uint4*>(a.w + static_cast<int64_t>(n) * (a.K / 2));
+#pragma unroll
+        for (int i = 0; i < GL_CPI; ++i) {
+            const int c = seg * 32 * GL_CPI + lane + 32 * i;
+            wv[i] = c < chunks ? __ldg(row + c) : make_uint4(0, 0, 0, 0);
+        }
+    };
+    // this CTA's channels [r0, r1) and this warp's items wid, wid + 8, ... of their (r1 - r0) * nseg items
+    const int r0 = static_cast<int>(static_cast<int64_t>(blockIdx.x) * a.N / gridDim.x);
+    const int r1 = static_cast<int>(static_cast<int64_t>(blockIdx.x + 1) * a.N / gridDim.x);
+    const int n_items = (r1 - r0) * nseg;
+    int* partial = reinterpret_cast<int*>(xs_long + a.K);   // one sum per item
+    uint4 bufA[GL_CPI], bufB[GL_CPI];   // two items in flight, both fetched before the dependency wait
+    auto item_row = [&](int j) { return r0 + (wid + 8 * j) / nseg; };
+    auto item_seg = [&](int j) { return (wid + 8 * j) % nseg; };
+    const int n_mine = (n_items - wid + 7) / 8;
+    if (0 < n_mine) load_item(item_row(0), item_seg(0), bufA);
+    if (1 < n_mine) load_item(item_row(1), item_seg(1), bufB);
+    pdl_launch_dependents();
+    pdl_wait();
+    int bs;
+    float sx;
+    // place of the 16 codes k = 16j .. 16j+15 of the row: block b = k / 128; offsets below 64 meet low nibbles
+    auto place = [&](int j) -> uint4* {
+        const int k = 16 * j, b = k >> 7, o = k & 127;
+        return (o < 64 ? lo : hi) + b * 4 + ((o & 63) >> 4);
+    };
+    if (FUSEQ) {
+        // the quantizer of quantize.cu for one row: max-abs, scale = amax / 7, inv = 7 / amax, codes by the magic add
+        const int n16 = a.K / 16;
+        const int64_t src = a.fuse_row_index ? static_cast<int64_t>(a.fuse_row_index[0]) : 0;
+        const uint4* xr = reinterpret_cast<const uint4*>(a.fuse_x + src * a.fuse_ldx);
+        float amax = 0.0f;
+        for (int c = tid; c < 2 * n16; c += 256) {
+            const uint4 v = __ldg(xr + c);
+            const __half2* h = reinterpret_cast<const __half2*>(&v);
+#pragma unroll
+            for (int q = 0; q < 4; ++q) {
+                const float2 f = __half22float2(__habs2(h[q]));
+                amax = fmaxf(amax, fmaxf(f.x, f.y));
+            }
+        }
+        amax = warp_max(amax);
+        if (lane == 0) red_f[wid] = amax;
+        __syncthreads();
+#pragma unroll
+        for (int w = 0; w < 8; ++w) amax = fmaxf(amax, red_f[w]);
+        float inv;
+        scale_of(amax, sx, inv);
+        int bias = 0;
+        for (int j = tid; j < n16; j += 256) {
+            uint32_t wd[4];
+#pragma unroll
+            for (int e = 0; e < 2; ++e) {
+                uint64_t p[4];
+                uint32_t t[8];
+                half8_to_pairs(__ldg(xr + 2 * j + e), p);
+#pragma unroll
+                for (int q = 0; q < 4; ++q) round_pair(p[q], inv, MAGIC, t[2 * q], t[2 * q + 1]);
+                wd[2 * e] = low_bytes(t[0], t[1], t[2], t[3]);
+                wd[2 * e + 1] = low_bytes(t[4], t[5], t[6], t[7]);
+            }
+            if (((16 * j) & 127) < 64) {   // these codes meet low weight nibbles
+#pragma unroll
+                for (int e = 0; e < 4; ++e) {
+                    bias = __dp4a(static_cast<int>(wd[e]), 0x01010101, bias);
+                    wd[e] = times16(wd[e]);
+                }
+            }
+            const uint4 out = make_uint4(wd[0], wd[1], wd[2], wd[3]);
+            *place(j) = out;
+            if (blockIdx.x == 0) reinterpret_cast<uint4*>(const_cast<int8_t*>(a.x8))[j] = out;
+        }
+        bias = warp_sum(bias);
+        if (lane == 0) red_i[wid] = bias;
+        __syncthreads();   // also: the codes are complete
+        bs = 0;
+#pragma unroll
+        for (int w = 0; w < 8; ++w) bs += red_i[w];
+        if (blockIdx.x == 0 && tid == 0) {
+            const_cast<int32_t*>(a.bias_sum)[0] = bs;
+            const_cast<float*>(a.act_scales)[0] = sx;
+        }
+    } else {
+        for (int j = tid; j < a.K / 16; j += 256) *place(j) = __ldg(reinterpret_cast<const uint4*>(a.x8) + j);
+        bs = a.bias_sum[0];
+        sx = a.act_scales[0];
+        __syncthreads();
+    }
+    auto do_item = [&](int it, uint4* wv) {
+        const int seg = item_seg(it);
+        int acc = 0;
+#pragma unroll
+        for (int i = 0; i < GL_CPI; ++i) {
+            const int c = seg * 32 * GL_CPI + lane + 32 * i;
+            if (c < chunks) {
+                const uint4 xl = lo[c], xh = hi[c];
+                const uint32_t w4[4] = {wv[i].x, wv[i].y, wv[i].z, wv[i].w};
+                const int l4[4] = {(int)xl.x, (int)xl.y, (int)xl.z, (int)xl.w};
+                const int h4[4] = {(int)xh.x, (int)xh.y, (int)xh.z, (int)xh.w};
+#pragma unroll
+                for (int q = 0; q < 4; ++q) {
+                    acc = __dp4a(l4[q], static_cast<int>(w4[q] & 0x0F0F0F0Fu), acc);
+                    acc = __dp4a(h4[q], static_cast<int>(w4[q] & 0xF0F0F0F0u), acc);
+                }
+            }
+        }
+        acc = warp_sum(acc);
+        if (lane == 0) partial[wid + 8 * it] = acc;
+        if (it + 2 < n_mine) load_item(item_row(it + 2), item_seg(it + 2), wv);
+    };
+    for (int it = 0; it < n_mine; it += 2) {
+        do_item(it, bufA);
+        if (it + 1 < n_mine) do_item(it + 1, bufB);
+    }
+    __syncthreads();
+    for (int r = tid; r < r1 - r0; r += 256) {
+        int acc = 0;
+        for (int sg = 0; sg < nseg; ++sg) acc += partial[r * nseg + sg];
+        const int n = r0 + r;
+        const int t = finish_acc(acc, bs);
+        store_out(a.out, n, a.out_dtype, dequant(t, sx, __half2float(a.w_scales[n])), t);
+    }
+}
+
+static void launch_gemv1_long(const LinearArgs& a, cudaStream_t s) {
+    const int blocks = sm_count() * 3;
+    const int need = (a.N + 7) / 8;
+    int grid = need < blocks ? need : blocks;
+    const int nseg = (a.K / 32 + 32 * GL_CPI - 1) / (32 * GL_CPI);
+    // shared memory: the codes (K <= MMA_FUSE_MAX_K bytes) and one partial sum per item of a CTA, within the default
+    // dynamic limit; a matrix with more channels than that allows per CTA gets more CTAs than are resident at once
+    const int rows_cap = (48 * 1024 - a.K) / (4 * nseg) - 1;
+    if ((a.N + grid - 1) / grid > rows_cap) grid = (a.N + rows_cap - 1) / rows_cap;
+    const size_t smem = static_cast<size_t>(a.K) + sizeof(int) * static_cast<size_t>((a.N + grid - 1) / grid + 1) * nseg;
+    cudaError_t e;
+    if (a.fuse_x) e = launch_dependent(w4a4_gemv1_long_kernel<true>, dim3(grid), dim3(256), smem, s, a);
+    else e = launch_dependent(w4a4_gemv1_long_kernel<false>, dim3(grid), dim3(256), smem, s, a);
+    if (e != cudaSuccess) note_cuda_error(e);
 }
 
 template <int CPL>
 static void launch_gemv1(const LinearArgs& a, cudaStream_t s) {
-    const int blocks = sm_count() * 3;
+    const int blocks = sm_count() * (a.w_up ? 2 : 3);   // resident CTAs per SM: the gated pair holds two register buffers
     const int need = (a.N + 7) / 8;
     const int grid = need < blocks ? need : blocks;
     cudaError_t e;
@@ -497,9 +684,9 @@ static sqap_status pick_path(const LinearArgs& a, uint32_t flags, LinearPath* pa
         const bool tc_ok = tcgen05_supports(a);
         const int w_tiles = (a.w_up ? 2 * a.N : a.N) / 128;
         // A handful of rows: the register-MMA streamer (its MMA rate holds up to ~16 rows; where the tensor-memory
-        // kernel has too few weight tiles to fill the SMs it stays ahead up to 32). One row of up to 4096 codes:
-        // the dp4a streamer that keeps the row in registers.
-        const bool one_row_in_registers = a.M == 1 && a.K / 32 <= 32 * 4;   // the dp4a streamer's best case
+        // kernel has too few weight tiles to fill the SMs it stays ahead up to 32). One row: the dp4a streamers
+        // (codes in registers up to 4096 of them; in shared memory up to 16384 for plain matrices).
+        const bool one_row_in_registers = a.M == 1 && (a.K / 32 <= 32 * 4 || (a.half == 64 && a.K <= MMA_FUSE_MAX_K && !a.w_up));
         const bool stream = mma_stream_supports(a) && !one_row_in_registers && (a.M <= 16 || w_tiles < 64);
         const bool gemv = !stream && a.M <= 8 && (!tc_ok || a.M <= 2 || (a.M <= 4 && w_tiles < 64));
         // CTA pairs fetch each token once per 256 weight rows: ahead from ~144 tokens on when there are enough pairs
@@ -525,6 +712,7 @@ static sqap_status run_gemm(const LinearArgs& a, LinearPath path, uint32_t flags
         const int chunks = a.K / 32;
         // rows up to 4096 codes: activation row in registers; longer rows would not amortise loading it
         if (a.M == 1 && chunks <= 32 * 4) launch_gemv1<4>(a, s);
+        else if (a.M == 1 && a.half == 64 && a.K <= MMA_FUSE_MAX_K && !a.w_up) launch_gemv1_long(a, s);
         else if (a.M == 1) launch_gemv<1>(a, s);
         else if (a.M == 2) launch_gemv<2>(a, s);
         else if (a.M <= 4) launch_gemv<4>(a, s);
@@ -602,7 +790,8 @@ sqap_status sqap_quantize_linear(const void* x, int M, int64_t ldx, const int32_
     st = pick_path(a, lflags, &path);
     if (st != SQAP_OK) return st;
     const bool one_plain_row = M == 1 && !(qflags & SQAP_Q_ROTATE);
-    if (one_plain_row && ((path == PATH_GEMV && a.K / 32 <= 32 * 4) || (path == PATH_MMA && a.K <= MMA_FUSE_MAX_K))) {
+    if (one_plain_row && ((path == PATH_GEMV && (a.K / 32 <= 32 * 4 || (a.half == 64 && a.K <= MMA_FUSE_MAX_K && !w_up))) ||
+                          (path == PATH_MMA && a.K <= MMA_FUSE_MAX_K))) {
         // one row, no rotation: the streamer quantizes the row itself (one kernel instead of two)
         a.fuse_x = static_cast<const __half*>(x);
         a.fuse_ldx = ldx;

@@ -258,7 +258,8 @@ def test_weight_quantizer_rejects_bad_arguments():
 # ------------------------------------------------------------------ linear: small and ragged shapes
 
 @pytest.mark.parametrize("M,N,K", [(1, 8, 32), (2, 128, 64), (7, 8, 512), (64, 512, 512), (65, 130, 96),
-                                   (9, 72, 11008), (130, 264, 1024), (300, 520, 256)])
+                                   (9, 72, 11008), (130, 264, 1024), (300, 520, 256), (1, 200, 11008), (1, 3000, 4224),
+                                   (1, 72, 16384), (1, 40, 20480)])
 def test_linear_small_shapes(M, N, K):
     x = wl.activations(20, M * 7 + K, M, K, max(1, K // 100), 20.0)
     wc = wl.weight_codes(20, N * 3 + K, N, K)
