@@ -867,15 +867,16 @@ def run_single_kernel(args):
     if args.kernel == "quantize":
         for i in range(args.steps):
             B.sqap_quantize_act(x, M, H, H, None, B.SQAP_Q_ROTATE if i % 2 == 0 else 0, q, sx)
-    elif args.kernel in ("gemm", "gemv", "stream", "midm", "downm", "swiglu"):
-        names = {"gemm": ("qkv",), "gemv": ("qkv",), "stream": ("qkv",), "midm": ("o",), "downm": ("down",),
-                 "swiglu": ("gate", "up")}[args.kernel]
+    elif args.kernel in ("gemm", "gemv", "gemvpair", "gemvlong", "stream", "midm", "downm", "swiglu"):
+        names = {"gemm": ("qkv",), "gemv": ("qkv",), "gemvpair": ("gate", "up"), "gemvlong": ("down",), "stream": ("qkv",),
+                 "midm": ("o",), "downm": ("down",), "swiglu": ("gate", "up")}[args.kernel]
         wts = wl.config4_weights(seed=4)
         ws = [B.sqap_pack_weights(np.ascontiguousarray(wts[n + "_codes"]), np.ascontiguousarray(wts[n + "_scales"]),
                                   wts[n + "_codes"].shape[0], wts[n + "_codes"].shape[1]) for n in names]
         # stream: one decode token per observation; midm / downm: one observation pruned to 160 rows (O projection on
         # the one-CTA-per-tile kernel; down projection, 11008 codes per row, on the cluster split-K kernel)
-        Mk = {"gemv": 1, "stream": N_OBS, "midm": 160, "downm": 160}.get(args.kernel, M)
+        # gemv / gemvpair / gemvlong: the single row of a decode step (QKV; gate + up; down with 11008 codes per row)
+        Mk = {"gemv": 1, "gemvpair": 1, "gemvlong": 1, "stream": N_OBS, "midm": 160, "downm": 160}.get(args.kernel, M)
         N = ws[0].N
         Kk = ws[0].K
         if Kk != H:
@@ -959,7 +960,7 @@ def main():
                     help="time every kernel of the path alone at the workload's shapes (one JSON table, no bench line)")
     ap.add_argument("--stack", action="store_true",
                     help="time configs[3] (32-layer stack: prefill + 7 decode tokens for one observation); own JSON line")
-    ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "stream", "midm", "downm", "quantize", "prune"],
+    ap.add_argument("--kernel", default=None, choices=["gemm", "swiglu", "gemv", "gemvpair", "gemvlong", "stream", "midm", "downm", "quantize", "prune"],
                     help="profiling aid: launch only this kernel --steps times (no bench line)")
     args = ap.parse_args()
     if args.gpus > 1 and "WORLD_SIZE" not in os.environ:
