@@ -176,6 +176,9 @@ class Path:
                              (self.x_host, self.scores_host, self.centers_host, self.xdec_host))
         self.d2h_bytes = sum(v.numel() * v.element_size() for v in (self.d1_host, self.ddec_host, self.kept_host))
         self.gemm_events = []
+        self.overlap_prune = True
+        self.side = t.cuda.Stream(device=device)
+        self.ev_fork, self.ev_join = t.cuda.Event(), t.cuda.Event()
         # second set of input / output device buffers: the end-to-end loop uploads step i+1 and downloads step i-1
         # while step i computes (intermediate buffers are shared: the compute stream runs the steps in order)
         self.io = [dict(x=self.x, scores=self.scores, centers=self.centers, xdec=self.xdec, d1=self.d1, ddec=self.ddec,
@@ -195,11 +198,29 @@ class Path:
         self.linear(self.h.data_ptr(), M, wl.FFN, wl.FFN, L.w["down"], None, d_out)
 
     def step(self, k: int = 0):
-        B, io = self.B, self.io[k]
-        self.layer(io["x"], M_FULL, self.layers[0], self.d)
-        # the criterion writes the kept rows as a source-row list; layer B's first quantizer reads them in place
-        B.sqap_prune_select(self.prune_params, io["scores"], io["centers"], ROWS_KEPT, io["kept"], self.nkept,
-                            self.row_index)
+        B, io, t = self.B, self.io[k], self.torch
+        H, L = wl.HIDDEN, self.layers[0]
+        # Layer A. The pruning criterion needs only the attention scores, which a model has once the layer's attention
+        # is done, so it does not have to wait for the layer's last linears: it is issued on a second stream after the
+        # gate / up projection and runs (16 small CTAs, latency-bound) beside the down projection's quantizer; layer B
+        # waits for both. It writes the kept rows as a source-row list, which layer B's first quantizer reads in place.
+        self.linear(io["x"].data_ptr(), M_FULL, H, H, L.w["qkv"], None, self.qkv, rotate=True)
+        self.linear(self.qkv.data_ptr() + 2 * 2 * H, M_FULL, H, wl.QKV, L.w["o"], None, self.o)   # V third of QKV
+        self.linear(self.o.data_ptr(), M_FULL, H, H, L.w["gate"], L.w["up"], self.h)
+        main = t.cuda.current_stream()
+        if self.overlap_prune:
+            self.ev_fork.record(main)
+            self.side.wait_event(self.ev_fork)
+            with t.cuda.stream(self.side):
+                B.sqap_prune_select(self.prune_params, io["scores"], io["centers"], ROWS_KEPT, io["kept"], self.nkept,
+                                    self.row_index)
+                self.ev_join.record(self.side)
+        self.linear(self.h.data_ptr(), M_FULL, wl.FFN, wl.FFN, L.w["down"], None, self.d)
+        if self.overlap_prune:
+            main.wait_event(self.ev_join)
+        else:
+            B.sqap_prune_select(self.prune_params, io["scores"], io["centers"], ROWS_KEPT, io["kept"], self.nkept,
+                                self.row_index)
         self.layer(io["x"], M_PRUNED, self.layers[1], io["d1"], row_index=self.row_index)
         self.layer(io["xdec"], N_OBS, self.layers[1], io["ddec"])
 
@@ -447,6 +468,7 @@ def run_ours(args):
     peaks = measured_peaks()
     sm_count = torch.cuda.get_device_properties(local_rank).multi_processor_count
     path = Path(torch, B, device, seed=4 + 1000 * rank, keep_host_weights=(rank == 0 and not args.no_parity_check))
+    path.overlap_prune = not args.serial_prune
     path.upload()
     torch.cuda.synchronize()
 
@@ -955,6 +977,8 @@ def main():
                     help="length in seconds of the second, sustained timed region (0: none)")
     ap.add_argument("--stub-backend", default=None, choices=["gloo"],
                     help="plumbing test: run the rank start-up, barriers and max-over-ranks timing around a CPU stub step")
+    ap.add_argument("--serial-prune", action="store_true",
+                    help="issue the pruning criterion on the main stream after layer A instead of beside its last quantizer")
     ap.add_argument("--no-graph", action="store_true", help="issue the step's launches eagerly instead of replaying a CUDA graph")
     ap.add_argument("--detail", action="store_true",
                     help="time every kernel of the path alone at the workload's shapes (one JSON table, no bench line)")
