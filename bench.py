@@ -738,6 +738,14 @@ def kernel_table(torch, B, peaks, device):
         fl = B.SQAP_Q_ROTATE if rot else 0
         us = graph_time_us(t, lambda i: B.sqap_quantize_act(xs[i % n], M, K, K, None, fl, q, sx), reps=max(n, 8))
         add("quantize_act" + ("+hadamard" if rot else ""), f"M={M} K={K}", "hbm", nb, us)
+        if M == M_FULL and K == H:
+            # the other granularities (sqap_quantize_act_ex); the tensor-wise form reads x twice (two launches), its
+            # algorithmic bytes stay those of one pass
+            mul = (t.rand(K, device=device, generator=gen) + 0.5).float()
+            for nm, f2, cm in (("channel-wise", fl, mul), ("tensor-wise", fl | B.SQAP_Q_PER_TENSOR, None)):
+                us = graph_time_us(t, lambda i: B.sqap_quantize_act_ex(xs[i % n], M, K, K, None, f2, cm, q, sx), reps=max(n, 8))
+                add("quantize_act_ex " + nm + ("+hadamard" if rot else ""), f"M={M} K={K}", "hbm", nb, us,
+                    note="two launches, x read twice" if cm is None else "")
         del xs
 
     # ---- gather (prune compaction) and the criterion

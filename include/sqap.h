@@ -136,8 +136,10 @@ sqap_status sqap_quantize_act(const void* x, int M, int K, int64_t ldx, const in
  *                      fp32(x) before the rotation and the max-abs (smoothing); put its reciprocal into the weights
  *                      with sqap_quantize_weights
  * Everything else (arguments, layout, rounding, SQAP_Q_ROTATE) is as in sqap_quantize_act, to which the call
- * falls through when neither extension is requested. K <= 16384. These two forms run in plain kernels (one CTA per
- * row, three launches for per-tensor): they are correct, not tuned.
+ * falls through when neither extension is requested. channel_mul is 16-byte aligned. Both forms run in the
+ * per-token quantizer's kernels; the tensor-wise form takes two launches (max-abs of the tensor, then the codes; x is
+ * read twice) and keeps the max-abs between them in a word of a 64-slot pool owned by the library, cleared on
+ * `stream`: up to 64 such calls may be in flight on different streams at once.
  */
 sqap_status sqap_quantize_act_ex(const void* x, int M, int K, int64_t ldx, const int32_t* row_index, uint32_t flags,
                                  const float* channel_mul, uint8_t* q_packed, float* scales, void* stream);

@@ -16,6 +16,8 @@
 //   SINK_EXPANDED  what the GEMM kernels multiply (linear.cuh): one int8 per code, codes that meet a low
 //                  weight nibble pre-multiplied by 16, plus the per-row sum of those codes. This skips the
 //                  expand pass when quantizer and linear run as one call (sqap_quantize_linear).
+#include <atomic>
+
 #include "quantize.cuh"
 
 namespace sqap {
@@ -40,6 +42,44 @@ __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
     uint64_t d;
     asm("sub.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
     return d;
+}
+
+__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
+    uint64_t d;
+    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
+    return d;
+}
+
+// The other granularities of sqap_quantize_act_ex, as template parameters of the same kernels:
+//   MUL   a static per-input-channel multiplier is applied to fp32(x) first ("channel-wise": smoothing)
+//   MODE  QM_TOKEN  one scale per row (the default);
+//         QM_AMAX   first pass of the tensor-wise form: only the max-abs, folded into one word with atomicMax
+//                   (the bits of a non-negative float order like the float);
+//         QM_GIVEN  second pass: every row is quantized with the max-abs found in that word.
+constexpr int QM_TOKEN = 0, QM_AMAX = 1, QM_GIVEN = 2;
+struct QuantEx {
+    const float* ch_mul;      // [K] or nullptr
+    unsigned* tensor_amax;    // the word of QM_AMAX / QM_GIVEN
+};
+__device__ __forceinline__ void fold_amax(unsigned* word, float amax) {
+    const unsigned bits = __float_as_uint(amax);
+    if (bits > *reinterpret_cast<volatile unsigned*>(word)) atomicMax(word, bits);   // most rows lose: skip their atomic
+}
+// Eight values k = 8c .. 8c+7 as packed pairs times their channel multipliers (each product rounded to fp32).
+__device__ __forceinline__ void scale_channels(uint64_t* p, const float* __restrict__ ch_mul, int c) {
+    const float4 m0 = __ldg(reinterpret_cast<const float4*>(ch_mul) + 2 * c), m1 = __ldg(reinterpret_cast<const float4*>(ch_mul) + 2 * c + 1);
+    p[0] = mul2(p[0], pk(m0.x, m0.y));
+    p[1] = mul2(p[1], pk(m0.z, m0.w));
+    p[2] = mul2(p[2], pk(m1.x, m1.y));
+    p[3] = mul2(p[3], pk(m1.z, m1.w));
+}
+__device__ __forceinline__ float absmax_pairs(const uint64_t* p, int n, float m) {
+    for (int i = 0; i < n; ++i) {
+        float a, b;
+        upk(p[i], a, b);
+        m = fmaxf(m, fmaxf(fabsf(a), fabsf(b)));
+    }
+    return m;
 }
 
 // Block-wide max of non-negative values; every thread gets the result. red: >= 32 floats of smem.
@@ -102,11 +142,11 @@ __device__ __forceinline__ void emit_chunk(const uint64_t* v, float inv, int c, 
 constexpr int QUANT_NIT = 8;
 constexpr int QUANT_THREADS = 256;
 
-template <int SINK, int G>
+template <int SINK, int G, int MODE = QM_TOKEN, bool MUL = false>
 __global__ void __launch_bounds__(QUANT_THREADS) quantize_rows_kernel(const __half* __restrict__ x, int M, int K,
                                                                       int64_t ldx,
                                                                       const int32_t* __restrict__ row_index,
-                                                                      QuantOut o) {
+                                                                      QuantOut o, QuantEx ex) {
     constexpr int ROWS = QUANT_THREADS / G, WARPS = G / 32;
     __shared__ float red_f[ROWS][WARPS];
     __shared__ int red_i[ROWS][WARPS];
@@ -119,28 +159,49 @@ __global__ void __launch_bounds__(QUANT_THREADS) quantize_rows_kernel(const __ha
     const uint4* xr = reinterpret_cast<const uint4*>(x + src * ldx);
     const int chunks = row_ok ? K / 8 : 0;
 
-    uint4 cache[QUANT_NIT];
-    __half2 m2 = __float2half2_rn(0.0f);
-    auto absmax = [&](const uint4& v) {
-        const __half2* h = reinterpret_cast<const __half2*>(&v);
-#pragma unroll
-        for (int i = 0; i < 4; ++i) m2 = __hmax2(m2, __habs2(h[i]));
+    // the row's values as packed fp32 pairs, channel multipliers applied (the same products in both passes)
+    auto pairs_of = [&](const uint4& raw, int c, uint64_t* p) {
+        half8_to_pairs(raw, p);
+        if constexpr (MUL) scale_channels(p, ex.ch_mul, c);
     };
+    uint4 cache[QUANT_NIT];
+    float amax = 0.0f;
+    if constexpr (MODE == QM_GIVEN) {
+        amax = __uint_as_float(*ex.tensor_amax);
+    } else {
+        __half2 m2 = __float2half2_rn(0.0f);
+        auto absmax = [&](const uint4& v, int c) {
+            if constexpr (MUL) {   // products are fp32
+                uint64_t p[4];
+                pairs_of(v, c, p);
+                amax = absmax_pairs(p, 4, amax);
+            } else {
+                const __half2* h = reinterpret_cast<const __half2*>(&v);
 #pragma unroll
-    for (int it = 0; it < QUANT_NIT; ++it) {
-        const int c = it * G + u;
-        if (c < chunks) cache[it] = __ldg(xr + c);
-    }
+                for (int i = 0; i < 4; ++i) m2 = __hmax2(m2, __habs2(h[i]));
+            }
+        };
 #pragma unroll
-    for (int it = 0; it < QUANT_NIT; ++it)
-        if (it * G + u < chunks) absmax(cache[it]);
-    for (int c = QUANT_NIT * G + u; c < chunks; c += G) absmax(__ldg(xr + c));
-    float amax = warp_max(fmaxf(__low2float(m2), __high2float(m2)));
-    if (WARPS > 1) {
-        if ((u & 31) == 0) red_f[g][u >> 5] = amax;
-        __syncthreads();
+        for (int it = 0; it < QUANT_NIT; ++it) {
+            const int c = it * G + u;
+            if (c < chunks) cache[it] = __ldg(xr + c);
+        }
 #pragma unroll
-        for (int w = 0; w < WARPS; ++w) amax = fmaxf(amax, red_f[g][w]);
+        for (int it = 0; it < QUANT_NIT; ++it)
+            if (it * G + u < chunks) absmax(cache[it], it * G + u);
+        for (int c = QUANT_NIT * G + u; c < chunks; c += G) absmax(__ldg(xr + c), c);
+        if constexpr (!MUL) amax = fmaxf(__low2float(m2), __high2float(m2));
+        amax = warp_max(amax);
+        if (WARPS > 1) {
+            if ((u & 31) == 0) red_f[g][u >> 5] = amax;
+            __syncthreads();
+#pragma unroll
+            for (int w = 0; w < WARPS; ++w) amax = fmaxf(amax, red_f[g][w]);
+        }
+        if constexpr (MODE == QM_AMAX) {
+            if (u == 0 && row_ok) fold_amax(ex.tensor_amax, amax);
+            return;
+        }
     }
     float scale, inv;
     scale_of(amax, scale, inv);
@@ -151,13 +212,14 @@ __global__ void __launch_bounds__(QUANT_THREADS) quantize_rows_kernel(const __ha
         const int c = it * G + u;
         if (c < chunks) {
             uint64_t p[4];
-            half8_to_pairs(cache[it], p);
+            if constexpr (MODE == QM_GIVEN) cache[it] = __ldg(xr + c);
+            pairs_of(cache[it], c, p);
             emit_chunk<SINK>(p, inv, c, o, row, K, bias);
         }
     }
     for (int c = QUANT_NIT * G + u; c < chunks; c += G) {
         uint64_t p[4];
-        half8_to_pairs(__ldg(xr + c), p);
+        pairs_of(__ldg(xr + c), c, p);
         emit_chunk<SINK>(p, inv, c, o, row, K, bias);
     }
     if (SINK == SINK_EXPANDED) {
@@ -173,12 +235,12 @@ __global__ void __launch_bounds__(QUANT_THREADS) quantize_rows_kernel(const __ha
     }
 }
 
-template <int SINK, int G>
+template <int SINK, int G, int MODE = QM_TOKEN, bool MUL = false>
 static void launch_plain(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, const QuantOut& o,
-                         cudaStream_t s) {
+                         cudaStream_t s, QuantEx ex = QuantEx{nullptr, nullptr}) {
     constexpr int ROWS = QUANT_THREADS / G;
-    const cudaError_t e = launch_dependent(quantize_rows_kernel<SINK, G>, dim3((M + ROWS - 1) / ROWS), dim3(QUANT_THREADS), 0, s,
-                                           x, M, K, ldx, row_index, o);
+    const cudaError_t e = launch_dependent(quantize_rows_kernel<SINK, G, MODE, MUL>, dim3((M + ROWS - 1) / ROWS),
+                                           dim3(QUANT_THREADS), 0, s, x, M, K, ldx, row_index, o, ex);
     if (e != cudaSuccess) note_cuda_error(e);
 }
 
@@ -190,7 +252,7 @@ static void launch_plain(const __half* x, int M, int K, int64_t ldx, const int32
 template <int E, int SINK>
 __global__ void __launch_bounds__(1024) quantize_rows_rotate_kernel(const __half* __restrict__ x, int K, int64_t ldx,
                                                                     const int32_t* __restrict__ row_index,
-                                                                    float norm, QuantOut o) {
+                                                                    float norm, QuantOut o, QuantEx ex, int mode) {
     extern __shared__ float sm[];  // K floats when K/E > 32, plus 32 for the reduction
     float* red = sm;
     float* buf = sm + 32;
@@ -223,6 +285,10 @@ __global__ void __launch_bounds__(1024) quantize_rows_rotate_kernel(const __half
             v[i] = f.x;
             v[i + 1] = f.y;
         }
+    }
+    if (ex.ch_mul) {   // channel-wise form: each product rounded to fp32 before the transform
+#pragma unroll
+        for (int i = 0; i < E; ++i) v[i] = __fmul_rn(v[i], __ldg(ex.ch_mul + t * E + i));
     }
     // register-local stages
 #pragma unroll
@@ -265,7 +331,15 @@ __global__ void __launch_bounds__(1024) quantize_rows_rotate_kernel(const __half
         v[j] = __fmul_rn(v[j], norm);
         amax = fmaxf(amax, fabsf(v[j]));
     }
-    amax = block_max(amax, red);
+    if (mode == QM_GIVEN) {
+        amax = __uint_as_float(*ex.tensor_amax);
+    } else {
+        amax = block_max(amax, red);
+        if (mode == QM_AMAX) {
+            if (t == 0) fold_amax(ex.tensor_amax, amax);
+            return;
+        }
+    }
     float scale, inv;
     scale_of(amax, scale, inv);
     if (t == 0) o.scales[row] = scale;
@@ -349,11 +423,11 @@ __device__ __forceinline__ void group_sync(int g) { asm volatile("bar.sync %0, 6
 // Persistent: a CTA walks rows blockIdx.x*4 + g, + 4*gridDim.x, ... . Each thread stages its own 128 input bytes
 // of the NEXT row with cp.async while the current row is transformed, so the HBM latency is off the critical path;
 // the staging slots are private to a thread (it alone writes and reads them), so they need no barrier.
-template <int SINK>
+template <int SINK, int MODE = QM_TOKEN, bool MUL = false>
 __global__ void __launch_bounds__(R4K_THREADS, 2) quantize_rotate4096_kernel(const __half* __restrict__ x, int M,
                                                                               int64_t ldx,
                                                                               const int32_t* __restrict__ row_index,
-                                                                              QuantOut o) {
+                                                                              QuantOut o, QuantEx ex) {
     extern __shared__ __align__(16) uint8_t smem_raw[];
     __shared__ float red_f[R4K_ROWS][2];
     __shared__ int red_i[R4K_ROWS][2];
@@ -386,8 +460,10 @@ __global__ void __launch_bounds__(R4K_THREADS, 2) quantize_rotate4096_kernel(con
         uint64_t P[32];
         cp_async_wait_all();
 #pragma unroll
-        for (int c = 0; c < 8; ++c)
+        for (int c = 0; c < 8; ++c) {
             half8_to_pairs(*reinterpret_cast<const uint4*>(stage + ((c ^ (u & 7)) << 4)), P + 4 * c);
+            if constexpr (MUL) scale_channels(P + 4 * c, ex.ch_mul, u * 8 + c);   // this thread's values are k = 64u ..
+        }
         prefetch(row + row_step);  // the values above are in registers: the slots are free again
         fwht64_pairs(P);           // h = 1 .. 32
 
@@ -411,16 +487,24 @@ __global__ void __launch_bounds__(R4K_THREADS, 2) quantize_rotate4096_kernel(con
         fwht64_pairs(P);  // h = 64 .. 2048
 
         float amax = 0.0f;
+        if constexpr (MODE != QM_GIVEN) {
 #pragma unroll
-        for (int i = 0; i < 32; ++i) {
-            float a, b;
-            upk(P[i], a, b);
-            amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+            for (int i = 0; i < 32; ++i) {
+                float a, b;
+                upk(P[i], a, b);
+                amax = fmaxf(amax, fmaxf(fabsf(a), fabsf(b)));
+            }
+            amax = warp_max(amax);
+            if ((u & 31) == 0) red_f[g][u >> 5] = amax;
         }
-        amax = warp_max(amax);
-        if ((u & 31) == 0) red_f[g][u >> 5] = amax;
         group_sync(g);  // also: every read of buf above is done before the bytes below overwrite it
-        amax = fmaxf(red_f[g][0], red_f[g][1]) * 0.015625f;  // exact
+        if constexpr (MODE == QM_GIVEN) amax = __uint_as_float(*ex.tensor_amax);
+        else amax = fmaxf(red_f[g][0], red_f[g][1]) * 0.015625f;  // exact
+        if constexpr (MODE == QM_AMAX) {
+            if (u == 0) fold_amax(ex.tensor_amax, amax);
+            group_sync(g);   // red_f is read: the next row may overwrite it
+            continue;
+        }
         float scale, inv;
         scale_of(amax, scale, inv);
         if (u == 0) o.scales[row] = scale;
@@ -465,76 +549,9 @@ __global__ void __launch_bounds__(R4K_THREADS, 2) quantize_rotate4096_kernel(con
     cp_async_wait_all();
 }
 
-// ---------------------------------------------------------------------------------------------
-// The other activation granularities the paper names (one scale per TENSOR; a per-CHANNEL multiplier applied
-// first), any row length, written for clarity rather than speed: one CTA per row, the row in shared memory as
-// fp32, Hadamard stages one after the other. mode 0: per-token; mode 1: only the row's max-abs, left in
-// scales[row]; mode 2: quantize with the max-abs found in scales[row] (the tensor's, after tensor_max_kernel).
-__global__ void __launch_bounds__(256) quantize_rows_general_kernel(const __half* __restrict__ x, int K, int64_t ldx,
-                                                                    const int32_t* __restrict__ row_index,
-                                                                    const float* __restrict__ ch_mul, int rotate,
-                                                                    float norm, int mode, uint8_t* __restrict__ q,
-                                                                    float* __restrict__ scales) {
-    extern __shared__ float row_f[];   // K floats
-    __shared__ float red[32];
-    const int row = blockIdx.x;
-    const int64_t src = row_index ? static_cast<int64_t>(row_index[row]) : static_cast<int64_t>(row);
-    const __half* xr = x + src * ldx;
-    for (int k = threadIdx.x; k < K; k += blockDim.x) {
-        float v = __half2float(xr[k]);
-        if (ch_mul) v = __fmul_rn(v, ch_mul[k]);
-        row_f[k] = v;
-    }
-    __syncthreads();
-    if (rotate) {
-        for (int h = 1; h < K; h <<= 1) {
-            for (int pr = threadIdx.x; pr < K / 2; pr += blockDim.x) {
-                const int j = (pr / h) * 2 * h + (pr % h);
-                const float a = row_f[j], b = row_f[j + h];
-                row_f[j] = __fadd_rn(a, b);
-                row_f[j + h] = __fsub_rn(a, b);
-            }
-            __syncthreads();
-        }
-        for (int k = threadIdx.x; k < K; k += blockDim.x) row_f[k] = __fmul_rn(row_f[k], norm);
-        __syncthreads();
-    }
-    float amax = 0.0f;
-    if (mode == 2) {
-        amax = scales[row];
-        __syncthreads();   // every thread has read it before thread 0 replaces it with the scale
-    } else {
-        for (int k = threadIdx.x; k < K; k += blockDim.x) amax = fmaxf(amax, fabsf(row_f[k]));
-        amax = block_max(amax, red);
-    }
-    if (mode == 1) {
-        if (threadIdx.x == 0) scales[row] = amax;
-        return;
-    }
-    float scale, inv;
-    scale_of(amax, scale, inv);
-    if (threadIdx.x == 0) scales[row] = scale;
-    uint32_t* qr = reinterpret_cast<uint32_t*>(q + static_cast<int64_t>(row) * (K / 2));
-    for (int c = threadIdx.x; c < K / 8; c += blockDim.x) {
-        uint32_t t[8];
-#pragma unroll
-        for (int i = 0; i < 8; ++i) t[i] = __float_as_uint(__fadd_rn(__fmul_rn(row_f[8 * c + i], inv), MAGIC8));
-        qr[c] = nibbles_of(low_bytes(t[0], t[1], t[2], t[3]), low_bytes(t[4], t[5], t[6], t[7]));
-    }
-}
-
-// scales[0 .. M) hold the rows' max-abs: replace every entry by their maximum.
-__global__ void __launch_bounds__(1024) tensor_max_kernel(float* __restrict__ scales, int M) {
-    __shared__ float red[32];
-    float m = 0.0f;
-    for (int i = threadIdx.x; i < M; i += blockDim.x) m = fmaxf(m, scales[i]);
-    m = block_max(m, red);
-    for (int i = threadIdx.x; i < M; i += blockDim.x) scales[i] = m;
-}
-
 template <int E, int SINK>
 static void launch_rotate(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, const QuantOut& o,
-                          cudaStream_t s) {
+                          cudaStream_t s, QuantEx ex = QuantEx{nullptr, nullptr}, int mode = QM_TOKEN) {
     const int T = K / E;
     const float norm = static_cast<float>(1.0 / sqrt(static_cast<double>(K)));
     const size_t smem = (32 + (T > 32 ? static_cast<size_t>(K) : 0)) * sizeof(float);
@@ -543,8 +560,24 @@ static void launch_rotate(const __half* x, int M, int K, int64_t ldx, const int3
         if (setup.run([](int*) { return set_max_dynamic_smem(quantize_rows_rotate_kernel<E, SINK>, (32 + 16384) * 4); }) != SQAP_OK)
             return;
     }
-    const cudaError_t e = launch_dependent(quantize_rows_rotate_kernel<E, SINK>, dim3(M), dim3(T), smem, s, x, K, ldx, row_index, norm, o);
+    const cudaError_t e = launch_dependent(quantize_rows_rotate_kernel<E, SINK>, dim3(M), dim3(T), smem, s, x, K, ldx, row_index, norm, o,
+                                           ex, mode);
     if (e != cudaSuccess) note_cuda_error(e);
+}
+
+template <int SINK, int MODE, bool MUL>
+static sqap_status launch_rotate4096(const __half* x, int M, int64_t ldx, const int32_t* row_index, const QuantOut& o,
+                                     const QuantEx& ex, cudaStream_t s) {
+    static PerDevice<int> setup;   // one per kernel instantiation
+    const sqap_status st = setup.run([](int*) { return set_max_dynamic_smem(quantize_rotate4096_kernel<SINK, MODE, MUL>, R4K_SMEM); });
+    if (st != SQAP_OK) return st;
+    int ctas = (M + R4K_ROWS - 1) / R4K_ROWS;
+    const int resident = 2 * sm_count();
+    if (ctas > resident) ctas = resident;
+    const cudaError_t e = launch_dependent(quantize_rotate4096_kernel<SINK, MODE, MUL>, dim3(ctas), dim3(R4K_THREADS), R4K_SMEM, s,
+                                           x, M, ldx, row_index, o, ex);
+    if (e != cudaSuccess) note_cuda_error(e);
+    return SQAP_OK;
 }
 
 template <int SINK>
@@ -552,15 +585,8 @@ static sqap_status launch_quantize(const __half* x, int M, int K, int64_t ldx, c
                                    const QuantOut& o, cudaStream_t s) {
     if (rotate) {
         if (K == R4K) {
-            static PerDevice<int> setup;
-            const sqap_status st = setup.run([](int*) { return set_max_dynamic_smem(quantize_rotate4096_kernel<SINK>, R4K_SMEM); });
+            const sqap_status st = launch_rotate4096<SINK, QM_TOKEN, false>(x, M, ldx, row_index, o, QuantEx{nullptr, nullptr}, s);
             if (st != SQAP_OK) return st;
-            int ctas = (M + R4K_ROWS - 1) / R4K_ROWS;
-            const int resident = 2 * sm_count();
-            if (ctas > resident) ctas = resident;
-            const cudaError_t e = launch_dependent(quantize_rotate4096_kernel<SINK>, dim3(ctas), dim3(R4K_THREADS), R4K_SMEM, s,
-                                                   x, M, ldx, row_index, o);
-            if (e != cudaSuccess) note_cuda_error(e);
         }
         // E elements per thread: 16 from K = 512 up (T = K/16 <= 1024), fewer for short rows so a full warp works
         else if (K >= 512) launch_rotate<16, SINK>(x, M, K, ldx, row_index, o, s);
@@ -595,6 +621,64 @@ sqap_status quantize_expanded(const __half* x, int M, int K, int64_t ldx, const 
     return launch_quantize<SINK_EXPANDED>(x, M, K, ldx, row_index, (flags & SQAP_Q_ROTATE) != 0, o, s);
 }
 
+// ---------------------------------------------------------------------------------------------
+// The other activation granularities the paper names (one scale per TENSOR; a per-CHANNEL multiplier applied
+// first) run in the same kernels as the per-token form (template parameters MODE / MUL above). The tensor-wise form
+// takes two launches: the first folds every row's max-abs into one word, the second quantizes with it (its reads
+// of x mostly hit L2). The word comes from a small pool in device memory, one slot per call in turn, cleared by a
+// 4-byte memset on the call's stream: calls in flight on different streams use different slots unless more than
+// TENSOR_SLOTS of them overlap; a captured CUDA graph keeps the slot it was captured with.
+constexpr int TENSOR_SLOTS = 64;
+__device__ unsigned g_tensor_amax[TENSOR_SLOTS];
+
+static unsigned* tensor_amax_slot() {
+    static PerDevice<unsigned*> base;
+    unsigned* const* p = nullptr;
+    if (base.run([](unsigned** out) {
+            void* addr = nullptr;
+            const cudaError_t e = cudaGetSymbolAddress(&addr, g_tensor_amax);
+            if (e != cudaSuccess) {
+                note_cuda_error(e);
+                return SQAP_ERR_CUDA;
+            }
+            *out = static_cast<unsigned*>(addr);
+            return SQAP_OK;
+        }, &p) != SQAP_OK)
+        return nullptr;
+    static std::atomic<unsigned> next{0};
+    return *p + next.fetch_add(1) % TENSOR_SLOTS;
+}
+
+template <int MODE, bool MUL>
+static sqap_status launch_ex(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, bool rotate, const QuantOut& o,
+                             const QuantEx& ex, cudaStream_t s) {
+    constexpr int SINK = SINK_NIBBLES;
+    if (rotate) {
+        if (K == R4K) {
+            const sqap_status st = launch_rotate4096<SINK, MODE, MUL>(x, M, ldx, row_index, o, ex, s);
+            if (st != SQAP_OK) return st;
+        } else if (K >= 512) launch_rotate<16, SINK>(x, M, K, ldx, row_index, o, s, ex, MODE);
+        else if (K == 256) launch_rotate<8, SINK>(x, M, K, ldx, row_index, o, s, ex, MODE);
+        else if (K == 128) launch_rotate<4, SINK>(x, M, K, ldx, row_index, o, s, ex, MODE);
+        else launch_rotate<2, SINK>(x, M, K, ldx, row_index, o, s, ex, MODE);
+    } else {
+        const int chunks = K / 8;
+        if (chunks <= 32 * QUANT_NIT) launch_plain<SINK, 32, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
+        else if (chunks <= 64 * QUANT_NIT) launch_plain<SINK, 64, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
+        else if (chunks <= 128 * QUANT_NIT) launch_plain<SINK, 128, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
+        else launch_plain<SINK, 256, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
+    }
+    count_launch();
+    return check_launch();
+}
+
+template <int MODE>
+static sqap_status launch_ex_mul(const __half* x, int M, int K, int64_t ldx, const int32_t* row_index, bool rotate,
+                                 const QuantOut& o, const QuantEx& ex, cudaStream_t s) {
+    return ex.ch_mul ? launch_ex<MODE, true>(x, M, K, ldx, row_index, rotate, o, ex, s)
+                     : launch_ex<MODE, false>(x, M, K, ldx, row_index, rotate, o, ex, s);
+}
+
 }  // namespace sqap
 
 extern "C" sqap_status sqap_quantize_act_ex(const void* x, int M, int K, int64_t ldx, const int32_t* row_index,
@@ -602,37 +686,30 @@ extern "C" sqap_status sqap_quantize_act_ex(const void* x, int M, int K, int64_t
                                             void* stream) {
     using namespace sqap;
     if (flags & ~(SQAP_Q_ROTATE | SQAP_Q_PER_TENSOR)) return SQAP_ERR_INVALID;
-    if (!(flags & SQAP_Q_PER_TENSOR) && !channel_mul)   // nothing extended asked for: the tuned per-token kernels
+    if (!(flags & SQAP_Q_PER_TENSOR) && !channel_mul)   // nothing extended asked for
         return sqap_quantize_act(x, M, K, ldx, row_index, flags, q_packed, scales, stream);
     const sqap_status st = quantize_check_args(x, M, K, ldx, flags & SQAP_Q_ROTATE);
     if (st != SQAP_OK || M == 0) return st;
     if (!q_packed || !scales) return SQAP_ERR_INVALID;
     if (!aligned16(q_packed)) return SQAP_ERR_ALIGN;
-    if ((reinterpret_cast<uintptr_t>(scales) & 3u) || (reinterpret_cast<uintptr_t>(channel_mul) & 3u)) return SQAP_ERR_ALIGN;
-    if (K > 16384) return SQAP_ERR_UNSUPPORTED;   // the row is held in shared memory as fp32
+    if (reinterpret_cast<uintptr_t>(scales) & 3u) return SQAP_ERR_ALIGN;
+    if (reinterpret_cast<uintptr_t>(channel_mul) & 15u) return SQAP_ERR_ALIGN;   // read 16 bytes at a time
     cudaStream_t s = static_cast<cudaStream_t>(stream);
-    const size_t smem = sizeof(float) * static_cast<size_t>(K);
-    if (smem > 48 * 1024) {
-        cudaError_t e = cudaFuncSetAttribute(quantize_rows_general_kernel, cudaFuncAttributeMaxDynamicSharedMemorySize,
-                                             static_cast<int>(smem));
-        if (e != cudaSuccess) {
-            note_cuda_error(e);
-            return SQAP_ERR_CUDA;
-        }
-    }
-    const int rotate = (flags & SQAP_Q_ROTATE) ? 1 : 0;
-    const float norm = static_cast<float>(1.0 / sqrt(static_cast<double>(K)));
+    const bool rotate = (flags & SQAP_Q_ROTATE) != 0;
     const __half* xh = static_cast<const __half*>(x);
-    if (flags & SQAP_Q_PER_TENSOR) {
-        quantize_rows_general_kernel<<<M, 256, smem, s>>>(xh, K, ldx, row_index, channel_mul, rotate, norm, 1, q_packed, scales);
-        tensor_max_kernel<<<1, 1024, 0, s>>>(scales, M);
-        quantize_rows_general_kernel<<<M, 256, smem, s>>>(xh, K, ldx, row_index, channel_mul, rotate, norm, 2, q_packed, scales);
-        count_launch(3);
-    } else {
-        quantize_rows_general_kernel<<<M, 256, smem, s>>>(xh, K, ldx, row_index, channel_mul, rotate, norm, 0, q_packed, scales);
-        count_launch();
+    QuantOut o{q_packed, nullptr, nullptr, scales, 64};
+    QuantEx ex{channel_mul, nullptr};
+    if (!(flags & SQAP_Q_PER_TENSOR)) return launch_ex_mul<QM_TOKEN>(xh, M, K, ldx, row_index, rotate, o, ex, s);
+    ex.tensor_amax = tensor_amax_slot();
+    if (!ex.tensor_amax) return SQAP_ERR_CUDA;
+    const cudaError_t e = cudaMemsetAsync(ex.tensor_amax, 0, sizeof(unsigned), s);
+    if (e != cudaSuccess) {
+        note_cuda_error(e);
+        return SQAP_ERR_CUDA;
     }
-    return check_launch();
+    const sqap_status s1 = launch_ex_mul<QM_AMAX>(xh, M, K, ldx, row_index, rotate, o, ex, s);
+    if (s1 != SQAP_OK) return s1;
+    return launch_ex_mul<QM_GIVEN>(xh, M, K, ldx, row_index, rotate, o, ex, s);
 }
 
 extern "C" sqap_status sqap_quantize_act(const void* x, int M, int K, int64_t ldx, const int32_t* row_index,

@@ -200,7 +200,8 @@ def test_weight_quantizer_bit_exact_and_feeds_the_linear(N, K, rotate):
 
 
 @pytest.mark.parametrize("M,K,rotate", [(12, 256, False), (12, 256, True), (37, 4096, True), (5, 11008, False),
-                                        (300, 512, True)])
+                                        (300, 512, True), (9, 64, True), (9, 128, True), (33, 4096, False),
+                                        (6, 20480, False), (1300, 4096, True), (3, 16384, True)])
 def test_quantizer_per_tensor_and_channel_multiplier(M, K, rotate):
     """sqap_quantize_act_ex in its two extra granularities (and both at once) against the oracle, with a row index
     list; then a smoothed linear end to end: activations times 1/d, weights times d, codes through the GEMM."""
