@@ -172,6 +172,7 @@ __global__ void __launch_bounds__(256) gather_rows_kernel(const __half* __restri
 // Every floating-point step is an explicitly rounded fp32 operation in a stated order (sqap.h), so
 // the scores, and with them the kept set, do not depend on this kernel's thread mapping.
 constexpr int ATTN_MAX_HEAD_DIM = 256;
+constexpr int ATTN_TILE = 256;   // most tokens whose keys are staged in shared memory at a time
 
 // 2^t for t <= 0: floor / fraction split, degree-9 Taylor polynomial of e^(f ln 2) in Horner form with
 // separately rounded multiplies and adds, exact scaling by 2^floor(t); 0 below -126.
@@ -191,7 +192,7 @@ __device__ __forceinline__ float exp2_neg(float t) {
 __global__ void __launch_bounds__(256) attention_scores_kernel(const __half* __restrict__ qkv, int64_t ldq, int rows,
                                                                int query_row, int visual_start, int n_visual,
                                                                int head_dim, int q_col0, int k_col0, float inv_sqrt_d,
-                                                               __half* __restrict__ out) {
+                                                               int tile_rows, __half* __restrict__ out) {
     __shared__ float qf[ATTN_MAX_HEAD_DIM];
     __shared__ float lg[PRUNE_MAX_VISUAL];
     __shared__ float red[32];
@@ -201,22 +202,42 @@ __global__ void __launch_bounds__(256) attention_scores_kernel(const __half* __r
     for (int d = threadIdx.x; d < head_dim; d += blockDim.x) qf[d] = __half2float(q[d]);
     __syncthreads();
     float m = -INFINITY;
-    for (int j = threadIdx.x; j < n_visual; j += blockDim.x) {
-        const __half* k = qkv + (static_cast<int64_t>(b) * rows + visual_start + j) * ldq + k_col0 + static_cast<int64_t>(h) * head_dim;
-        float acc = 0.0f;
-        for (int d = 0; d < head_dim; d += 8) {   // head_dim % 8 == 0: 16-byte loads, sums in d order
-            const uint4 raw = __ldg(reinterpret_cast<const uint4*>(k + d));
-            const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
-#pragma unroll
-            for (int i = 0; i < 4; ++i) {
-                const float2 kv = __half22float2(h2[i]);
-                acc = __fadd_rn(acc, __fmul_rn(qf[d + 2 * i], kv.x));
-                acc = __fadd_rn(acc, __fmul_rn(qf[d + 2 * i + 1], kv.y));
-            }
+    // A thread owns a token (its sum runs in d order, as defined), but a token's key row is only head_dim * 2 bytes of
+    // a much longer row of the QKV output: read straight from global memory, the 32 lanes of a load would touch 32
+    // separate rows. So the CTA first copies the keys of up to 256 tokens into shared memory with coalesced 16-byte
+    // asynchronous copies (consecutive threads take consecutive chunks of a row), rows padded by 16 bytes so that the
+    // row-per-thread reads that follow are free of bank conflicts.
+    extern __shared__ __align__(16) uint8_t ktile[];
+    const int cpr = head_dim / 8, row_stride = head_dim * 2 + 16;
+    for (int j0 = 0; j0 < n_visual; j0 += tile_rows) {
+        const int tile = min(tile_rows, n_visual - j0);
+        const __half* kbase = qkv + (static_cast<int64_t>(b) * rows + visual_start + j0) * ldq + k_col0 + static_cast<int64_t>(h) * head_dim;
+        for (int i = threadIdx.x; i < tile * cpr; i += blockDim.x) {
+            const int r = i / cpr, c = i - r * cpr;
+            const uint32_t dst = static_cast<uint32_t>(__cvta_generic_to_shared(ktile + r * row_stride + 16 * c));
+            asm volatile("cp.async.cg.shared.global [%0], [%1], 16;" ::"r"(dst), "l"(kbase + static_cast<int64_t>(r) * ldq + 8 * c) : "memory");
         }
-        const float l = __fmul_rn(acc, inv_sqrt_d);
-        lg[j] = l;
-        m = fmaxf(m, l);
+        asm volatile("cp.async.commit_group;" ::: "memory");
+        asm volatile("cp.async.wait_group 0;" ::: "memory");
+        __syncthreads();
+        for (int jj = threadIdx.x; jj < tile; jj += blockDim.x) {
+            const uint8_t* k = ktile + jj * row_stride;
+            float acc = 0.0f;
+            for (int d = 0; d < head_dim; d += 8) {
+                const uint4 raw = *reinterpret_cast<const uint4*>(k + 2 * d);
+                const __half2* h2 = reinterpret_cast<const __half2*>(&raw);
+#pragma unroll
+                for (int i = 0; i < 4; ++i) {
+                    const float2 kv = __half22float2(h2[i]);
+                    acc = __fadd_rn(acc, __fmul_rn(qf[d + 2 * i], kv.x));
+                    acc = __fadd_rn(acc, __fmul_rn(qf[d + 2 * i + 1], kv.y));
+                }
+            }
+            const float l = __fmul_rn(acc, inv_sqrt_d);
+            lg[j0 + jj] = l;
+            m = fmaxf(m, l);
+        }
+        __syncthreads();   // the tile is read: the next one may overwrite it
     }
     // block max (exact, order-free)
 #pragma unroll
@@ -256,9 +277,18 @@ extern "C" sqap_status sqap_attention_scores(const void* qkv, int64_t ldq, int b
     if (head_dim % 8 != 0 || ldq % 8 != 0 || k_col0 % 8 != 0 || !aligned16(qkv)) return SQAP_ERR_ALIGN;
     const float inv_sqrt_d = static_cast<float>(1.0 / sqrt(static_cast<double>(head_dim)));
     dim3 grid(n_heads, batch);
-    attention_scores_kernel<<<grid, 256, 0, static_cast<cudaStream_t>(stream)>>>(
+    // 256 tokens per tile when the grid fits the SMs three CTAs deep (one pass over a 16 x 16 patch grid); half that
+    // otherwise, so that more CTAs are resident and the grid runs as one wave
+    const int tile_rows = static_cast<int64_t>(n_heads) * batch <= 3 * sm_count() ? ATTN_TILE : ATTN_TILE / 2;
+    const size_t smem = static_cast<size_t>(tile_rows) * (head_dim * 2 + 16);
+    if (smem > 48 * 1024) {
+        static PerDevice<int> setup;   // the limit covers the longest supported head
+        const sqap_status st = setup.run([](int*) { return set_max_dynamic_smem(attention_scores_kernel, ATTN_TILE * (ATTN_MAX_HEAD_DIM * 2 + 16)); });
+        if (st != SQAP_OK) return st;
+    }
+    attention_scores_kernel<<<grid, 256, smem, static_cast<cudaStream_t>(stream)>>>(
         static_cast<const __half*>(qkv), ldq, rows, query_row, visual_start, n_visual, head_dim, q_col0, k_col0, inv_sqrt_d,
-        static_cast<__half*>(scores_out));
+        tile_rows, static_cast<__half*>(scores_out));
     count_launch();
     return check_launch();
 }

@@ -649,7 +649,10 @@ def test_prune_fps_worked_example():
     assert kept[0, :5].tolist() == [0, 15, 119, 240, 255]
 
 
-@pytest.mark.parametrize("batch,rows,vs,nv,H,D", [(2, 40, 3, 24, 4, 32), (3, 288, 1, 256, 32, 128), (1, 70, 0, 64, 2, 8)])
+@pytest.mark.parametrize("batch,rows,vs,nv,H,D", [(2, 40, 3, 24, 4, 32), (3, 288, 1, 256, 32, 128), (1, 70, 0, 64, 2, 8),
+                                                  (1, 620, 4, 600, 2, 256),      # three key tiles, the longest head
+                                                  (16, 300, 2, 288, 32, 32),     # 512 CTAs: half-size tiles, ragged
+                                                  (15, 80, 0, 64, 32, 64)])
 def test_attention_scores_bit_exact_and_feed_the_criterion(batch, rows, vs, nv, H, D):
     """sqap_attention_scores against the oracle (fp16 bits), then scores -> criterion on the device against the
     oracle's kept rows: quantizer output -> attention -> pruning without leaving the GPU."""
