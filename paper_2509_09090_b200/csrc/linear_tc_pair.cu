@@ -170,12 +170,32 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
     // Everything above is independent of the kernel before this one in the stream; its output (the activations,
-    // their sums and scales) is read, and this kernel's output written, only from here on.
-    pdl_wait();
-
+    // their sums and scales) is read, and this kernel's output written, only after pdl_wait() below. The packed
+    // weights are immutable, so the producer fetches the first stages' weights BEFORE that wait: they travel while
+    // the quantizer before this kernel is still running.
     if (warp == 0) {
         // ---------------- TMA producer (one lane)
         if (lane == 0) {
+            // packed weights of stage ks of the tile whose weight rows (this CTA's half) start at n0: rows of 128
+            // bytes (both 128-code blocks of the stage) in one box
+            auto load_weights = [&](int st, int ks, int n0) {
+                const uint32_t wp = base + OFF_WP + st * (2 * WPH_BYTES);
+                if (a.swiglu) {
+                    tma_load_2d(wp, &tm_w, ks * (BK / 2), n0 / 2, full(st));
+                    tma_load_2d(wp + WPH_BYTES, &tm_w_up, ks * (BK / 2), n0 / 2, full(st));
+                } else {
+                    tma_load_2d(wp, &tm_w, ks * (BK / 2), n0, full(st));
+                }
+            };
+            uint32_t early = 0;   // stages of the first tile whose weights are already on their way
+            if (pair < total_tiles) {
+                early = static_cast<uint32_t>(k_steps < S ? k_steps : S);
+                for (uint32_t ks = 0; ks < early; ++ks) {
+                    mbar_expect_tx(full(ks), w_tx);
+                    load_weights(static_cast<int>(ks), static_cast<int>(ks), (pair % a.n_tiles) * (2 * BM) + static_cast<int>(rank) * BM);
+                }
+            }
+            pdl_wait();
             uint32_t it = 0;
             for (int tile = pair; tile < total_tiles && !failed; tile += n_pairs) {
                 const int n0 = (tile % a.n_tiles) * (2 * BM) + static_cast<int>(rank) * BM;
@@ -183,18 +203,13 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
                 for (int ks = 0; ks < k_steps; ++ks, ++it) {
                     const int s = it % S;
                     const uint32_t ph = (it / S) & 1u;
-                    if (!mbar_wait(done(s), ph ^ 1u, abort_flag) || !mbar_wait(wp_empty(s), ph ^ 1u, abort_flag)) { failed = true; break; }
-                    mbar_expect_tx(full(s), w_tx);
+                    if (it >= early) {
+                        if (!mbar_wait(done(s), ph ^ 1u, abort_flag) || !mbar_wait(wp_empty(s), ph ^ 1u, abort_flag)) { failed = true; break; }
+                        mbar_expect_tx(full(s), w_tx);
+                        load_weights(s, ks, n0);
+                    }
                     if (rank == 0) mbar_expect_tx(x_full(s), x_tx);
                     const uint32_t x_bar = map_to_cta(x_full(s), 0);
-                    // packed weights: rows of 128 bytes (both 128-code blocks of the stage) in one box
-                    const uint32_t wp = base + OFF_WP + s * (2 * WPH_BYTES);
-                    if (a.swiglu) {
-                        tma_load_2d(wp, &tm_w, ks * (BK / 2), n0 / 2, full(s));
-                        tma_load_2d(wp + WPH_BYTES, &tm_w_up, ks * (BK / 2), n0 / 2, full(s));
-                    } else {
-                        tma_load_2d(wp, &tm_w, ks * (BK / 2), n0, full(s));
-                    }
 #pragma unroll
                     for (int h = 0; h < 2; ++h)
                         tma_load_2d_pair(base + OFF_X + (2 * s + h) * XH_BYTES, &tm_x, ks * BK + h * BKH, m0, x_bar);
@@ -212,6 +227,7 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
             }
         }
     } else if (warp == 1) {
+        pdl_wait();
         // ---------------- MMA issuer (leader CTA): the whole warp walks the loop, one elected lane issues
         if (rank == 0) {
             const uint32_t issue = elect_one();
@@ -243,6 +259,8 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
             }
         }
     } else if (warp < 6) {
+        // (no dependency wait here: these warps touch shared and tensor memory only, and may unpack the weights that
+        // were fetched early while the kernel before this one still runs)
         // ---------------- unpack warps: thread = one tensor-memory lane = one weight row of the tile
         const int quad = warp & 3;                 // the lane quadrant this warp may write
         const int L = quad * 32 + lane;            // tensor-memory lane
@@ -286,6 +304,7 @@ w4a4_tc_pair_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_const
             }
         }
     } else {
+        pdl_wait();
         // ---------------- epilogue warps: warp % 4 selects the 32-lane quadrant of tensor memory
         const int quad = warp & 3;
         const int row = quad * 32 + lane;

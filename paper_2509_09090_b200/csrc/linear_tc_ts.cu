@@ -138,28 +138,42 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
     const uint32_t tmem_base = *tmem_slot;
     bool failed = false;
     // Everything above is independent of the kernel before this one in the stream; its output (the activations,
-    // their sums and scales) is read, and this kernel's output written, only from here on.
-    pdl_wait();
-
+    // their sums and scales) is read, and this kernel's output written, only after pdl_wait() below. The packed
+    // weights are immutable, so the producer fetches the first stages' weights BEFORE that wait: they travel while
+    // the quantizer before this kernel is still running.
     if (warp == 0) {
         // ---------------- TMA producer: the whole warp walks the loop, one elected lane issues
         const uint32_t issue = elect_one();
+        // packed weights of stage ks of the tile at weight row n0: rows of 128 bytes (both 128-code blocks) in one box
+        auto load_weights = [&](int st, int ks, int n0) {
+            const uint32_t wp = w_addr(st);
+            if (a.swiglu) {
+                tma_load_2d_if(wp, &tm_w, ks * (BK / 2), n0 / 2, full(st), issue);
+                tma_load_2d_if(wp + W_BYTES / 2, &tm_w_up, ks * (BK / 2), n0 / 2, full(st), issue);
+            } else {
+                tma_load_2d_if(wp, &tm_w, ks * (BK / 2), n0, full(st), issue);
+            }
+        };
+        uint32_t early = 0;   // stages of the first tile whose weights are already on their way
+        if (static_cast<int>(blockIdx.x) < total_tiles) {
+            early = static_cast<uint32_t>(k_steps < S ? k_steps : S);
+            for (uint32_t ks = 0; ks < early; ++ks) {
+                mbar_expect_tx_if(full(ks), stage_tx, issue);   // the whole stage: the activations follow after the wait
+                load_weights(static_cast<int>(ks), static_cast<int>(ks), (static_cast<int>(blockIdx.x) % a.n_tiles) * BM);
+            }
+        }
+        pdl_wait();
         uint32_t it = 0;
         int s = 0;
         uint32_t ph = 0;
         for (int tile = blockIdx.x; tile < total_tiles && !failed; tile += gridDim.x) {
             const int n0 = (tile % a.n_tiles) * BM, m0 = (tile / a.n_tiles) * a.BN;
             for (int ks = 0; ks < k_steps; ++ks, ++it) {
-                const bool ok = mbar_wait(done(s), ph ^ 1u, abort_flag) && mbar_wait(wp_empty(s), ph ^ 1u, abort_flag);
-                if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
-                mbar_expect_tx_if(full(s), stage_tx, issue);
-                // packed weights: rows of 128 bytes (both 128-code blocks of the stage) in one box
-                const uint32_t wp = w_addr(s);
-                if (a.swiglu) {
-                    tma_load_2d_if(wp, &tm_w, ks * (BK / 2), n0 / 2, full(s), issue);
-                    tma_load_2d_if(wp + W_BYTES / 2, &tm_w_up, ks * (BK / 2), n0 / 2, full(s), issue);
-                } else {
-                    tma_load_2d_if(wp, &tm_w, ks * (BK / 2), n0, full(s), issue);
+                if (it >= early) {
+                    const bool ok = mbar_wait(done(s), ph ^ 1u, abort_flag) && mbar_wait(wp_empty(s), ph ^ 1u, abort_flag);
+                    if (!__all_sync(0xffffffffu, ok)) { failed = true; break; }
+                    mbar_expect_tx_if(full(s), stage_tx, issue);
+                    load_weights(s, ks, n0);
                 }
 #pragma unroll
                 for (int h = 0; h < 2; ++h) tma_load_2d_if(x_addr(s, h), &tm_x, ks * BK + h * BKH, m0, full(s), issue);
@@ -174,6 +188,7 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
             }
         }
     } else if (warp == 1) {
+        pdl_wait();
         // ---------------- MMA issuer: the whole warp walks the loop, one elected lane issues
         {
             const uint32_t issue = elect_one();
@@ -208,6 +223,8 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
             }
         }
     } else if (warp < 6) {
+        // (no dependency wait here: these warps touch shared and tensor memory only, and may unpack the weights that
+        // were fetched early while the kernel before this one still runs)
         // ---------------- unpack warps: thread = one tensor-memory lane = one weight row of the tile
         const int quad = warp & 3;                 // the lane quadrant this warp may write
         const int L = quad * 32 + lane;            // tensor-memory lane
@@ -287,6 +304,7 @@ w4a4_tc_ts_kernel(const __grid_constant__ CUtensorMap tm_w, const __grid_constan
             if (j >= U) j = 0;
         }
     } else {
+        pdl_wait();
         // ---------------- epilogue warps: warp % 4 selects the 32-lane quadrant of tensor memory
         const int quad = warp & 3;
         const int row = quad * 32 + lane;
