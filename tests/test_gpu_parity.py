@@ -270,6 +270,32 @@ def test_linear_small_shapes(M, N, K):
         check_linear(x, wc, ws, flags_list=[B.SQAP_L_FORCE_GEMV])
 
 
+def _random_linear_shapes(n, seed):
+    """Seeded shapes across every regime of the dispatcher (single rows, a handful, mid-size, many tiles; short and
+    long rows; K % 128 == 0 or not), small enough for the oracle."""
+    rng = np.random.default_rng(seed)
+    ms = [1, 1, 1, 2, 3, 5, 8, 9, 16, 17, 31, 32, 33, 63, 64, 100, 143, 144, 200, 320, 321, 511, 512, 600]
+    ks = [32, 64, 96, 128, 256, 384, 1024, 2048, 4096, 4224, 8192, 11008, 12288, 16384]
+    out = []
+    while len(out) < n:
+        M, K = int(rng.choice(ms)), int(rng.choice(ks))
+        N = 8 * int(rng.integers(1, 400))
+        if M * N * K > 4e8:
+            continue
+        out.append((M, N, K, bool(rng.integers(0, 2)), bool(rng.integers(0, 2)) and (K & (K - 1)) == 0 and K >= 64))
+    return out
+
+
+@pytest.mark.parametrize("M,N,K,swiglu,rotate", _random_linear_shapes(40, 2509))
+def test_linear_random_shapes_through_the_dispatcher(M, N, K, swiglu, rotate):
+    """Whatever kernel the dispatcher picks for a shape: int32 accumulators bit-exact, outputs within tolerance, the
+    fused call identical to the two-call route."""
+    x = wl.activations(27, M + N + K, M, K, max(1, K // 100), 20.0)
+    g = (wl.weight_codes(27, N + K, N, K), wl.weight_scales(27, N + K, N, mult=0.5))
+    u = (wl.weight_codes(27, N + K + 1, N, K), wl.weight_scales(27, N + K + 1, N, mult=0.5)) if swiglu else None
+    check_linear(x, g[0], g[1], rotate=rotate, up=u, flags_list=[0])
+
+
 @pytest.mark.parametrize("M,N,K,swiglu", [(16, 128, 128, False), (9, 8, 256, False), (257, 130, 384, False),
                                           (144, 320, 1024, False), (700, 200, 512, False), (40, 192, 512, True),
                                           (300, 64, 256, True), (513, 448, 1152, True), (17, 1088, 11008, False),
