@@ -73,6 +73,13 @@ __device__ __forceinline__ void scale_channels(uint64_t* p, const float* __restr
     p[2] = mul2(p[2], pk(m1.x, m1.y));
     p[3] = mul2(p[3], pk(m1.z, m1.w));
 }
+// A 16-byte load that does not take a line of L1 (the channel-wise form streams x once and wants the multipliers,
+// which every row re-reads, to stay there).
+__device__ __forceinline__ uint4 ld_once(const uint4* p) {
+    uint4 v;
+    asm volatile("ld.global.nc.L1::no_allocate.v4.u32 {%0,%1,%2,%3}, [%4];" : "=r"(v.x), "=r"(v.y), "=r"(v.z), "=r"(v.w) : "l"(p));
+    return v;
+}
 __device__ __forceinline__ float absmax_pairs(const uint64_t* p, int n, float m) {
     for (int i = 0; i < n; ++i) {
         float a, b;
@@ -164,7 +171,11 @@ __global__ void __launch_bounds__(QUANT_THREADS) quantize_rows_kernel(const __ha
         half8_to_pairs(raw, p);
         if constexpr (MUL) scale_channels(p, ex.ch_mul, c);
     };
-    uint4 cache[QUANT_NIT];
+    // held between the two passes: the raw fp16 chunks, or (channel-wise form) the fp32 products of half as many
+    // chunks per thread (twice the threads per row), so that neither the products nor the multipliers are formed twice
+    constexpr int NIT = MUL ? QUANT_NIT / 2 : QUANT_NIT;
+    uint4 cache[MUL ? 1 : NIT];
+    uint64_t prod[MUL ? NIT : 1][4];
     float amax = 0.0f;
     if constexpr (MODE == QM_GIVEN) {
         amax = __uint_as_float(*ex.tensor_amax);
@@ -181,15 +192,28 @@ __global__ void __launch_bounds__(QUANT_THREADS) quantize_rows_kernel(const __ha
                 for (int i = 0; i < 4; ++i) m2 = __hmax2(m2, __habs2(h[i]));
             }
         };
+        if constexpr (MUL) {
+            uint4 raw[NIT];
 #pragma unroll
-        for (int it = 0; it < QUANT_NIT; ++it) {
-            const int c = it * G + u;
-            if (c < chunks) cache[it] = __ldg(xr + c);
+            for (int it = 0; it < NIT; ++it)
+                if (it * G + u < chunks) raw[it] = ld_once(xr + it * G + u);
+#pragma unroll
+            for (int it = 0; it < NIT; ++it)
+                if (it * G + u < chunks) {
+                    pairs_of(raw[it], it * G + u, prod[it]);
+                    amax = absmax_pairs(prod[it], 4, amax);
+                }
+        } else {
+#pragma unroll
+            for (int it = 0; it < NIT; ++it) {
+                const int c = it * G + u;
+                if (c < chunks) cache[it] = __ldg(xr + c);
+            }
+#pragma unroll
+            for (int it = 0; it < NIT; ++it)
+                if (it * G + u < chunks) absmax(cache[it], it * G + u);
         }
-#pragma unroll
-        for (int it = 0; it < QUANT_NIT; ++it)
-            if (it * G + u < chunks) absmax(cache[it], it * G + u);
-        for (int c = QUANT_NIT * G + u; c < chunks; c += G) absmax(__ldg(xr + c), c);
+        for (int c = NIT * G + u; c < chunks; c += G) absmax(__ldg(xr + c), c);
         if constexpr (!MUL) amax = fmaxf(__low2float(m2), __high2float(m2));
         amax = warp_max(amax);
         if (WARPS > 1) {
@@ -208,16 +232,19 @@ __global__ void __launch_bounds__(QUANT_THREADS) quantize_rows_kernel(const __ha
     if (u == 0 && row_ok) o.scales[row] = scale;
     int bias = 0;
 #pragma unroll
-    for (int it = 0; it < QUANT_NIT; ++it) {
+    for (int it = 0; it < NIT; ++it) {
         const int c = it * G + u;
         if (c < chunks) {
-            uint64_t p[4];
-            if constexpr (MODE == QM_GIVEN) cache[it] = __ldg(xr + c);
-            pairs_of(cache[it], c, p);
-            emit_chunk<SINK>(p, inv, c, o, row, K, bias);
+            if constexpr (MUL && MODE != QM_GIVEN) {
+                emit_chunk<SINK>(prod[it], inv, c, o, row, K, bias);
+            } else {
+                uint64_t p[4];
+                pairs_of(MODE == QM_GIVEN ? __ldg(xr + c) : cache[MUL ? 0 : it], c, p);
+                emit_chunk<SINK>(p, inv, c, o, row, K, bias);
+            }
         }
     }
-    for (int c = QUANT_NIT * G + u; c < chunks; c += G) {
+    for (int c = NIT * G + u; c < chunks; c += G) {
         uint64_t p[4];
         pairs_of(__ldg(xr + c), c, p);
         emit_chunk<SINK>(p, inv, c, o, row, K, bias);
@@ -663,9 +690,10 @@ static sqap_status launch_ex(const __half* x, int M, int K, int64_t ldx, const i
         else launch_rotate<2, SINK>(x, M, K, ldx, row_index, o, s, ex, MODE);
     } else {
         const int chunks = K / 8;
-        if (chunks <= 32 * QUANT_NIT) launch_plain<SINK, 32, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
-        else if (chunks <= 64 * QUANT_NIT) launch_plain<SINK, 64, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
-        else if (chunks <= 128 * QUANT_NIT) launch_plain<SINK, 128, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
+        constexpr int nit = MUL ? QUANT_NIT / 2 : QUANT_NIT;   // chunks a thread holds between the passes
+        if (chunks <= 32 * nit) launch_plain<SINK, 32, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
+        else if (chunks <= 64 * nit) launch_plain<SINK, 64, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
+        else if (chunks <= 128 * nit) launch_plain<SINK, 128, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
         else launch_plain<SINK, 256, MODE, MUL>(x, M, K, ldx, row_index, o, s, ex);
     }
     count_launch();
