@@ -44,11 +44,6 @@ __device__ __forceinline__ uint64_t sub2(uint64_t a, uint64_t b) {
     return d;
 }
 
-__device__ __forceinline__ uint64_t mul2(uint64_t a, uint64_t b) {
-    uint64_t d;
-    asm("mul.rn.f32x2 %0, %1, %2;" : "=l"(d) : "l"(a), "l"(b));
-    return d;
-}
 
 // The other granularities of sqap_quantize_act_ex, as template parameters of the same kernels:
 //   MUL   a static per-input-channel multiplier is applied to fp32(x) first ("channel-wise": smoothing)
@@ -65,13 +60,19 @@ __device__ __forceinline__ void fold_amax(unsigned* word, float amax) {
     const unsigned bits = __float_as_uint(amax);
     if (bits > *reinterpret_cast<volatile unsigned*>(word)) atomicMax(word, bits);   // most rows lose: skip their atomic
 }
-// Eight values k = 8c .. 8c+7 as packed pairs times their channel multipliers (each product rounded to fp32).
+// Eight values k = 8c .. 8c+7 as packed pairs times their channel multipliers (each product rounded to fp32). Scalar
+// __fmul_rn on purpose: it is never contracted with an add that follows (the first butterfly stage, when the row is
+// rotated), whereas a packed multiply followed by a packed add was seen to become a fused multiply-add even with
+// explicit rounding modes.
 __device__ __forceinline__ void scale_channels(uint64_t* p, const float* __restrict__ ch_mul, int c) {
     const float4 m0 = __ldg(reinterpret_cast<const float4*>(ch_mul) + 2 * c), m1 = __ldg(reinterpret_cast<const float4*>(ch_mul) + 2 * c + 1);
-    p[0] = mul2(p[0], pk(m0.x, m0.y));
-    p[1] = mul2(p[1], pk(m0.z, m0.w));
-    p[2] = mul2(p[2], pk(m1.x, m1.y));
-    p[3] = mul2(p[3], pk(m1.z, m1.w));
+    const float m[8] = {m0.x, m0.y, m0.z, m0.w, m1.x, m1.y, m1.z, m1.w};
+#pragma unroll
+    for (int i = 0; i < 4; ++i) {
+        float a, b;
+        upk(p[i], a, b);
+        p[i] = pk(__fmul_rn(a, m[2 * i]), __fmul_rn(b, m[2 * i + 1]));
+    }
 }
 // A 16-byte load that does not take a line of L1 (the channel-wise form streams x once and wants the multipliers,
 // which every row re-reads, to stay there).
