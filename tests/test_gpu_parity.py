@@ -242,6 +242,30 @@ def test_quantizer_per_tensor_and_channel_multiplier(M, K, rotate):
     handle.close()
 
 
+def test_per_tensor_quantizer_calls_in_flight_on_two_streams():
+    """The tensor's max-abs travels between the two launches of a per-tensor call in a word of a pool owned by the
+    library; calls on different streams must not see each other's word. Two streams, different tensors (one with a
+    far larger max-abs), many calls each, issued alternately without synchronising in between."""
+    M, K = 96, 1024
+    xa = wl.activations(63, 1, M, K, 4, 30.0)
+    xb = (wl.activations(63, 2, M, K, 4, 30.0).astype(np.float32) * np.float32(0.01)).astype(np.float16)
+    ref = [oracle.quantize_act(bits(v), per_tensor=True) for v in (xa, xb)]
+    dev = [G.to_dev(v) for v in (xa, xb)]
+    streams = [torch.cuda.Stream(), torch.cuda.Stream()]
+    reps = 12
+    q = [[torch.empty(M, K // 2, dtype=torch.uint8, device="cuda") for _ in range(reps)] for _ in range(2)]
+    s = [[torch.empty(M, dtype=torch.float32, device="cuda") for _ in range(reps)] for _ in range(2)]
+    torch.cuda.synchronize()
+    for r in range(reps):
+        for i in range(2):
+            B.sqap_quantize_act_ex(dev[i], M, K, K, None, B.SQAP_Q_PER_TENSOR, None, q[i][r], s[i][r], stream=streams[i])
+    torch.cuda.synchronize()
+    for i in range(2):
+        for r in range(reps):
+            assert np.array_equal(q[i][r].cpu().numpy(), ref[i][0]), (i, r)
+            assert np.array_equal(s[i][r].cpu().numpy(), ref[i][1]), (i, r)
+
+
 def test_weight_quantizer_rejects_bad_arguments():
     w = torch.zeros(8 * 96, dtype=torch.float16, device="cuda")
     c = torch.zeros(8 * 96, dtype=torch.int8, device="cuda")
