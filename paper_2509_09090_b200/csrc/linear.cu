@@ -404,9 +404,15 @@ __global__ void __launch_bounds__(256, SWIGLU ? 2 : 3) w4a4_gemv1_kernel(LinearA
             }
         }
     } else {
-        for (int n = gw; n < a.N; n += step) {
-            if (n != gw) load_item(n, A0, A1);
-            do_item(n, A0, A1);
+        // plain matrix: the two halves of an item are single rows n, n + W, ...; each half is refilled with the row two
+        // places further as soon as it has been used, so a load is always in flight while the other half is multiplied
+        for (int n = gw; n < a.N; n += 2 * W) {
+            finish(n, dot(A0), 0);
+            if (n + 2 * W < a.N) load_row(a.w, n + 2 * W, A0);
+            if (n + W < a.N) {
+                finish(n + W, dot(A1), 0);
+                if (n + 3 * W < a.N) load_row(a.w, n + 3 * W, A1);
+            }
         }
     }
 }
